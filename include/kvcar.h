@@ -1,0 +1,235 @@
+/*
+ * kvcar.h -- C ABI of the KV-CAR decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA, attention over a paged KV cache
+ * that stores per-layer autoencoder latents of K and V instead of K and V, plus
+ * a per-layer/per-head table that lets a head read the adjacent lower layer's
+ * cached K or V and store nothing (paper: Sec. "Network Architecture"; Eq. 1 for
+ * the attention itself; Eq. 3 for the cache-size model).
+ *
+ * Conventions
+ *   - Every call returns a kvcar_status; nothing throws or aborts across the ABI.
+ *     kvcar_last_error() gives a human-readable reason for the last failure.
+ *   - "HOST" / "DEVICE" beside a pointer says where the memory lives.
+ *   - All DEVICE memory is owned by the caller: the library reports the sizes it
+ *     needs (kvcar_required_bytes), receives three buffers (kvcar_bind_memory)
+ *     and never allocates or frees device memory itself.  Buffers must be
+ *     256-byte aligned and must outlive the context.
+ *   - Kernels are launched on the cudaStream_t the caller passes (as void*; 0 is
+ *     the default stream).  Calls are asynchronous with respect to the device;
+ *     host-side bookkeeping (page table mirror, sequence lengths) is updated
+ *     immediately, so all calls on one context must use one stream or be
+ *     ordered by the caller.
+ *   - Element type of q/k/v/out and of the cache rows is config.storage
+ *     (float or bfloat16); all accumulation is fp32.
+ *   - Matrices are row-major; autoencoder weights are [out][in].
+ *   - There is no CPU fallback: without a CUDA device the launching calls fail
+ *     with KVCAR_ERR_CUDA.
+ */
+#ifndef KVCAR_H
+#define KVCAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvcar_ctx kvcar_ctx;
+
+typedef enum {
+    KVCAR_OK = 0,
+    KVCAR_ERR_INVALID_ARG = 1,   /* bad pointer, index, size or alignment            */
+    KVCAR_ERR_STATE = 2,         /* call not allowed in the context's current state  */
+    KVCAR_ERR_OOM_PAGES = 3,     /* page pool exhausted; nothing was changed         */
+    KVCAR_ERR_WORKSPACE = 4,     /* bound buffers too small for the request          */
+    KVCAR_ERR_UNSUPPORTED = 5,   /* shape outside what the kernels handle            */
+    KVCAR_ERR_CUDA = 6,          /* a CUDA runtime/driver call failed                */
+    KVCAR_ERR_DEVICE_TIMEOUT = 7 /* a bounded device-side wait ran out               */
+} kvcar_status;
+
+typedef enum { KVCAR_F32 = 0, KVCAR_BF16 = 1 } kvcar_dtype;
+typedef enum { KVCAR_K = 0, KVCAR_V = 1 } kvcar_which;
+
+/* kernel families (kvcar_set_kernel) */
+typedef enum {
+    KVCAR_KERNEL_AUTO = 0,    /* tensor-core kernel where the shape allows, else generic */
+    KVCAR_KERNEL_GENERIC = 1, /* fp32-FMA kernels (any supported shape, both dtypes)     */
+    KVCAR_KERNEL_TENSOR = 2   /* tcgen05/TMEM fused kernel (bf16 storage only)           */
+} kvcar_kernel;
+
+/* flags of kvcar_decode_attention */
+#define KVCAR_INCLUDE_CURRENT_EXACT 1u /* also attend to the current token through its exact K/V */
+
+#define KVCAR_MAX_BATCH 512    /* sequences per launching call   */
+#define KVCAR_MAX_KV_HEADS 32
+#define KVCAR_MAX_Q_HEADS 128
+#define KVCAR_MAX_HEAD_DIM 128
+
+typedef struct {
+    int32_t n_layers;
+    int32_t n_q_heads;         /* query heads; multiple of n_kv_heads (grouped-query attention) */
+    int32_t n_kv_heads;
+    int32_t head_dim;
+    int32_t page_tokens;       /* tokens per cache page                                          */
+    int32_t max_seqs;          /* sequence ids are 0 .. max_seqs-1                               */
+    int32_t max_pages;         /* physical pages shared by all sequences (and all layers)       */
+    int32_t max_pages_per_seq; /* longest sequence = max_pages_per_seq * page_tokens tokens     */
+    int32_t storage;           /* kvcar_dtype of q/k/v/out and of cache rows                    */
+} kvcar_config;
+
+/*
+ * One autoencoder (encoder + decoder) for the K or the V of one layer, as the
+ * paper describes it (Sec. "Network Architecture"): FC(in_dim -> hidden),
+ * BatchNorm over the hidden features with stored statistics, LeakyReLU,
+ * FC(hidden -> latent); the decoder mirrors it (latent -> hidden -> in_dim).
+ * in_dim must equal (#heads the layer stores for this K/V) * head_dim: the
+ * autoencoder spans exactly the heads that are cached (a reused head is never
+ * encoded).  All pointers are HOST float arrays, read during the call only.
+ * *_bn is [4][hidden] = gamma, beta, running mean, running variance.
+ */
+typedef struct {
+    int32_t in_dim, hidden, latent;
+    float leaky_slope, bn_eps;
+    const float *enc_w1, *enc_b1, *enc_bn, *enc_w2, *enc_b2; /* [hidden][in_dim], [hidden], [4][hidden], [latent][hidden], [latent] */
+    const float *dec_w1, *dec_b1, *dec_bn, *dec_w2, *dec_b2; /* [hidden][latent], [hidden], [4][hidden], [in_dim][hidden], [in_dim] */
+} kvcar_ae;
+
+/* ---- set-up ------------------------------------------------------------- */
+
+/* Create a context (host bookkeeping only; touches no device).  Errors:
+ * INVALID_ARG for non-positive sizes, n_q_heads not a multiple of n_kv_heads, or
+ * limits above the KVCAR_MAX_* constants. */
+kvcar_status kvcar_create(const kvcar_config *cfg, kvcar_ctx **out_ctx);
+kvcar_status kvcar_destroy(kvcar_ctx *ctx);
+
+/*
+ * Cross-layer head reuse (Sec. "Network Architecture", last paragraph: "certain
+ * key and value heads in layer N reuse key and value heads from the previous
+ * layer N-1").  src_k/src_v: HOST int32 [n_layers * n_kv_heads]; entry
+ * (layer, head) is -1 if the head keeps its own cache rows, else the index of
+ * the head of layer-1 whose cached K (resp. V) it reads.  Chains are legal and
+ * resolve transitively.  Layer 0 must be all -1.  Only before kvcar_bind_memory
+ * (ERR_STATE after) and before any kvcar_set_autoencoder.  Default: all -1.
+ */
+kvcar_status kvcar_set_reuse_map(kvcar_ctx *ctx, const int32_t *src_k, const int32_t *src_v);
+
+/*
+ * Install the autoencoder of (layer, which).  A (layer, which) without one
+ * stores the raw rows of its stored heads (uncompressed layer).  Only before
+ * kvcar_bind_memory.  Errors: INVALID_ARG if in_dim does not match the stored
+ * heads or a pointer is NULL.
+ */
+kvcar_status kvcar_set_autoencoder(kvcar_ctx *ctx, int32_t layer, int32_t which, const kvcar_ae *ae);
+
+/* Sizes (bytes) of the three DEVICE buffers the context needs:
+ * pool = all cache pages of all layers + the current-token rows;
+ * weights = packed autoencoder weights and per-layer tables;
+ * workspace = page table, sequence lengths, split-KV partial results, staging. */
+kvcar_status kvcar_required_bytes(kvcar_ctx *ctx, size_t *pool, size_t *weights, size_t *workspace);
+
+/* Hand over the three DEVICE buffers (256-byte aligned, at least the required
+ * sizes), upload weights and tables on `stream`, and freeze the reuse map and
+ * autoencoders.  Must be called once, with the target device current. */
+kvcar_status kvcar_bind_memory(kvcar_ctx *ctx, void *pool, size_t pool_bytes, void *weights, size_t weights_bytes,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/* Choose the kernel family used by the launching calls (default AUTO). */
+kvcar_status kvcar_set_kernel(kvcar_ctx *ctx, int32_t kernel);
+
+/* ---- sequences and pages -------------------------------------------------- */
+
+/* Open / close a sequence id (0 <= seq < max_seqs).  Closing returns its pages:
+ * the page released last is handed out first; a fresh pool hands out 0,1,2,... */
+kvcar_status kvcar_seq_open(kvcar_ctx *ctx, int32_t seq);
+kvcar_status kvcar_seq_close(kvcar_ctx *ctx, int32_t seq);
+
+/* Make sure pages exist for positions seq_len .. seq_len+n_tokens-1 of each
+ * listed sequence (pages are taken in list order).  All or nothing: on
+ * ERR_OOM_PAGES no page has been taken.  Host-side only; the device copy of the
+ * page table is brought up to date by the next launching call. */
+kvcar_status kvcar_reserve(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens);
+
+/* ---- the hot path --------------------------------------------------------- */
+
+/*
+ * Encoder + append (Sec. "Network Architecture": "an encoder layer is added
+ * after the generation of key and value tokens ... reduces them to a lower
+ * dimension d ... a 1 x d vector is appended to the KV cache").
+ * k, v: DEVICE [n_seqs][n_tokens][n_kv_heads*head_dim] new rows (all heads;
+ * columns of reused heads are ignored).  For each sequence the stored heads'
+ * slices are encoded (or copied, for an uncompressed layer), rounded to the
+ * storage type and written at logical positions seq_len .. seq_len+n_tokens-1
+ * (pages are reserved first; on ERR_OOM_PAGES nothing is written).  The last
+ * token's exact rows are also kept as the layer's "current token".  seq_len is
+ * NOT changed: call kvcar_advance once per step after all layers.
+ * seqs: HOST int32 [n_seqs], distinct open sequences, n_seqs <= KVCAR_MAX_BATCH.
+ */
+kvcar_status kvcar_encode_append(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                 int32_t n_tokens, const void *k, const void *v, void *stream);
+
+/* seq_len += n_tokens for the listed sequences (host mirror now, device copy in
+ * stream order). */
+kvcar_status kvcar_advance(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens, void *stream);
+
+/*
+ * Decoder + attention (Sec. "Network Architecture": cached latents "are passed
+ * through two decoders, expanding them to (l-1) x D ... then concatenated with
+ * the current 1 x D key and value vectors"; Eq. 1 per head).
+ * q: DEVICE [n_seqs][n_q_heads][head_dim]; out: DEVICE, same shape.
+ * For each sequence and query head i (KV head g = i / (n_q_heads/n_kv_heads)):
+ * resolve g through the reuse table for K and for V separately, restore the
+ * root layer's cached rows 0 .. seq_len-1 with that layer's decoder, take the
+ * head's 64-wide slice, and compute softmax(q K^T / sqrt(head_dim)) V.  With
+ * KVCAR_INCLUDE_CURRENT_EXACT the exact current-token K/V written by this
+ * step's kvcar_encode_append of the root layer joins the attended set.
+ * A sequence with nothing to attend to yields zeros.
+ */
+kvcar_status kvcar_decode_attention(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                    const void *q, void *out, uint32_t flags, void *stream);
+
+/*
+ * The same two calls for one layer with HOST buffers: copies k, v, q (each
+ * n_tokens = 1) to the device, runs kvcar_encode_append then
+ * kvcar_decode_attention, and copies `out` back, all on `stream`.  Returns
+ * after enqueuing; synchronise the stream before reading out_host.  Host
+ * buffers should be page-locked for the copies to be asynchronous.
+ */
+kvcar_status kvcar_step_layer_host(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                   const void *k_host, const void *v_host, const void *q_host, void *out_host,
+                                   uint32_t flags, void *stream);
+
+/* ---- observability ---------------------------------------------------------- */
+
+/* Reuse table resolution of (layer, kv_head): the layer and head whose cache
+ * rows are read, and the 64-wide column slot of that head among the root
+ * layer's stored heads (ascending head order). */
+kvcar_status kvcar_debug_resolve(kvcar_ctx *ctx, int32_t layer, int32_t kv_head, int32_t which,
+                                 int32_t *root_layer, int32_t *root_head, int32_t *slot);
+/* Physical page and pool row of a logical token (must lie in a reserved page). */
+kvcar_status kvcar_debug_locate(kvcar_ctx *ctx, int32_t seq, int32_t token, int32_t *page, int64_t *row);
+kvcar_status kvcar_seq_len(kvcar_ctx *ctx, int32_t seq, int32_t *len);
+/* Placement of one layer's K or V rows inside the pool buffer: byte offset of
+ * row 0, bytes between rows, and elements per row (0 if the layer stores none). */
+kvcar_status kvcar_pool_layout(kvcar_ctx *ctx, int32_t layer, int32_t which, size_t *offset, size_t *row_pitch,
+                               int32_t *width);
+/* Bytes one cached token occupies over all layers: as configured, and with
+ * neither autoencoders nor reuse (Eq. 3 per token and sequence). */
+kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *ctx, double *compressed, double *uncompressed);
+/* Algorithmic work of one kvcar_decode_attention call on `layer` per cached
+ * token: latent bytes read and floating-point operations (decoder + attention),
+ * following the reuse map (each distinct source layer is read and passed
+ * through its first decoder layer once). */
+kvcar_status kvcar_layer_work_per_token(kvcar_ctx *ctx, int32_t layer, double *bytes, double *flops);
+/* Number of kernels the library has launched so far on this context. */
+kvcar_status kvcar_launch_count(kvcar_ctx *ctx, int64_t *count);
+/* Synchronise `stream` and report any asynchronous CUDA error or device-side
+ * bounded-wait timeout recorded since the last call. */
+kvcar_status kvcar_sync_status(kvcar_ctx *ctx, void *stream);
+const char *kvcar_last_error(kvcar_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVCAR_H */

@@ -1,0 +1,777 @@
+// Host runtime and C ABI of the KV-CAR decode path: configuration, reuse-map
+// resolution, page allocator, weight packing, per-layer device tables and the
+// launch logic.  See include/kvcar.h for the contract of every entry point.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "kvcar_internal.h"
+#include "kvcar_tc.h"
+
+using namespace kvcar;
+
+namespace {
+
+struct AEHost {
+    bool set = false;
+    int in_dim = 0, hidden = 0, latent = 0;
+    float slope = 0.f, eps = 0.f;
+    std::vector<float> enc_w1, enc_b1, enc_bn, enc_w2, enc_b2, dec_w1, dec_b1, dec_bn, dec_w2, dec_b2;
+};
+
+struct Resolved {
+    int root_layer, root_head, slot;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct kvcar_ctx {
+    kvcar_config cfg{};
+    int elem = 4;  // bytes per storage element
+    std::vector<int32_t> src[2];
+    std::vector<AEHost> ae;  // [layer*2 + which]
+    bool bound = false;
+    int kernel = KVCAR_KERNEL_AUTO;
+
+    // pages
+    std::vector<int32_t> free_pages;
+    std::vector<std::vector<int32_t>> table;
+    std::vector<int32_t> len;
+    std::vector<char> open;
+    std::vector<int4> pending;  // device table updates not yet enqueued
+    bool table_dirty_all = false;
+
+    // device buffers and layout
+    char *pool = nullptr, *weights = nullptr, *ws = nullptr;
+    std::vector<size_t> pool_off, cur_off;  // [layer*2+which]
+    std::vector<int> width;                 // elements per row
+    size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
+    size_t plan_off = 0, enc_off = 0;       // inside weights
+    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0;  // inside workspace
+    int max_chunks = 0, chunk_tokens = 128;
+    int max_d = 0, max_m = 0, max_in = 0;
+    std::vector<LayerPlan> plans_host;
+    TcState tc;
+
+    int64_t launches = 0;
+    std::string err;
+};
+
+namespace {
+
+kvcar_status fail(kvcar_ctx *c, kvcar_status s, const std::string &msg) {
+    if (c) c->err = msg;
+    return s;
+}
+kvcar_status cuda_fail(kvcar_ctx *c, cudaError_t e, const char *what) {
+    return fail(c, KVCAR_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+std::vector<int> stored_heads(const kvcar_ctx *c, int layer, int which) {
+    std::vector<int> h;
+    for (int i = 0; i < c->cfg.n_kv_heads; ++i)
+        if (c->src[which][layer * c->cfg.n_kv_heads + i] < 0) h.push_back(i);
+    return h;
+}
+
+Resolved resolve(const kvcar_ctx *c, int layer, int head, int which) {
+    const int hkv = c->cfg.n_kv_heads;
+    int l = layer, h = head;
+    while (c->src[which][l * hkv + h] >= 0) {
+        h = c->src[which][l * hkv + h];
+        --l;
+    }
+    int slot = 0;
+    for (int i = 0; i < h; ++i)
+        if (c->src[which][l * hkv + i] < 0) ++slot;
+    return {l, h, slot};
+}
+
+int stored_width(const kvcar_ctx *c, int layer, int which) {
+    const AEHost &a = c->ae[layer * 2 + which];
+    if (a.set) return a.latent;
+    return (int)stored_heads(c, layer, which).size() * c->cfg.head_dim;
+}
+
+void compute_layout(kvcar_ctx *c) {
+    const kvcar_config &g = c->cfg;
+    const int nl = g.n_layers;
+    const size_t rows = (size_t)g.max_pages * g.page_tokens;
+    const int W = g.n_kv_heads * g.head_dim;
+    c->pool_off.assign(nl * 2, 0);
+    c->cur_off.assign(nl * 2, 0);
+    c->width.assign(nl * 2, 0);
+    size_t off = 0;
+    c->max_d = c->max_m = c->max_in = 0;
+    for (int i = 0; i < nl * 2; ++i) {
+        c->width[i] = stored_width(c, i / 2, i % 2);
+        c->pool_off[i] = off;
+        off = align_up(off + rows * c->width[i] * c->elem, 256);
+        const AEHost &a = c->ae[i];
+        if (a.set) {
+            c->max_d = std::max(c->max_d, a.latent);
+            c->max_m = std::max(c->max_m, a.hidden);
+            c->max_in = std::max(c->max_in, a.in_dim);
+        } else {
+            c->max_in = std::max(c->max_in, c->width[i]);
+        }
+    }
+    for (int i = 0; i < nl * 2; ++i) {
+        c->cur_off[i] = off;
+        off = align_up(off + (size_t)g.max_seqs * W * c->elem, 256);
+    }
+    c->pool_bytes = off;
+
+    // weights: per (layer, which) packed arrays, then LayerPlan[nl], EncPlan[nl*2]
+    size_t w = 0;
+    for (int i = 0; i < nl * 2; ++i) {
+        const AEHost &a = c->ae[i];
+        if (!a.set) continue;
+        size_t mats = (size_t)a.in_dim * a.hidden + (size_t)a.hidden * a.latent;  // one half (enc or dec)
+        w = align_up(w + 2 * mats * c->elem, 256);                                 // transposed enc + dec
+        w = align_up(w + (size_t)(4 * a.hidden + a.latent + a.in_dim) * sizeof(float), 256);  // s,t x2, b2 x2
+        if (g.storage == KVCAR_BF16) w = align_up(w + mats * 2, 256);             // K-major decoder copies
+    }
+    c->plan_off = w;
+    w = align_up(w + (size_t)nl * sizeof(LayerPlan), 256);
+    c->enc_off = w;
+    w = align_up(w + (size_t)nl * 2 * sizeof(EncPlan), 256);
+    c->weights_bytes = w;
+
+    // workspace
+    c->chunk_tokens = 128;
+    const int cap = g.max_pages_per_seq * g.page_tokens;
+    c->max_chunks = (cap + c->chunk_tokens - 1) / c->chunk_tokens;
+    size_t s = 0;
+    c->bt_off = s;
+    s = align_up(s + (size_t)g.max_seqs * g.max_pages_per_seq * 4, 256);
+    c->len_off = s;
+    s = align_up(s + (size_t)g.max_seqs * 4, 256);
+    c->status_off = s;
+    s = align_up(s + 256, 256);
+    c->part_off = s;
+    const int nb = std::min(g.max_seqs, KVCAR_MAX_BATCH);
+    s = align_up(s + (size_t)nb * c->max_chunks * g.n_q_heads * (g.head_dim + 2) * sizeof(float), 256);
+    c->stage_off = s;
+    s = align_up(s + (size_t)nb * (2 * W + 2 * g.n_q_heads * g.head_dim) * c->elem + 4 * 256, 256);
+    c->ws_bytes = s;
+}
+
+void put_elems(char *dst, const float *src, size_t n, int dtype) {
+    if (dtype == KVCAR_F32) {
+        memcpy(dst, src, n * 4);
+    } else {
+        __nv_bfloat16 *d = reinterpret_cast<__nv_bfloat16 *>(dst);
+        for (size_t i = 0; i < n; ++i) d[i] = __float2bfloat16_rn(src[i]);
+    }
+}
+
+// transposed copy: src [rows][cols] -> dst [cols][rows]
+void put_transposed(char *dst, const float *src, int rows, int cols, int dtype) {
+    std::vector<float> t((size_t)rows * cols);
+    for (int r = 0; r < rows; ++r)
+        for (int cc = 0; cc < cols; ++cc) t[(size_t)cc * rows + r] = src[(size_t)r * cols + cc];
+    put_elems(dst, t.data(), t.size(), dtype);
+}
+
+// bias + BatchNorm(inference) as one scale/shift per feature
+void fuse_bn(const std::vector<float> &b1, const std::vector<float> &bn, int m, float eps, float *s, float *t) {
+    for (int j = 0; j < m; ++j) {
+        double gamma = bn[j], beta = bn[m + j], mean = bn[2 * m + j], var = bn[3 * m + j];
+        double sc = gamma / std::sqrt(var + (double)eps);
+        s[j] = (float)sc;
+        t[j] = (float)(((double)b1[j] - mean) * sc + beta);
+    }
+}
+
+bool check_seqs(kvcar_ctx *c, const int32_t *seqs, int n) {
+    if (!seqs || n <= 0 || n > KVCAR_MAX_BATCH) return false;
+    for (int i = 0; i < n; ++i) {
+        if (seqs[i] < 0 || seqs[i] >= c->cfg.max_seqs || !c->open[seqs[i]]) return false;
+    }
+    return true;
+}
+
+kvcar_status reserve_pages(kvcar_ctx *c, const int32_t *seqs, int n, int n_tokens) {
+    const int P = c->cfg.page_tokens;
+    size_t need_total = 0;
+    std::vector<int> need(n);
+    for (int i = 0; i < n; ++i) {
+        int s = seqs[i];
+        int want = (c->len[s] + n_tokens + P - 1) / P;
+        if (want > c->cfg.max_pages_per_seq) return fail(c, KVCAR_ERR_OOM_PAGES, "sequence exceeds max_pages_per_seq");
+        need[i] = std::max(0, want - (int)c->table[s].size());
+        need_total += need[i];
+    }
+    if (need_total > c->free_pages.size()) return fail(c, KVCAR_ERR_OOM_PAGES, "page pool exhausted");
+    for (int i = 0; i < n; ++i) {
+        int s = seqs[i];
+        for (int k = 0; k < need[i]; ++k) {
+            int page = c->free_pages.back();
+            c->free_pages.pop_back();
+            c->pending.push_back(make_int4(0, s, (int)c->table[s].size(), page));
+            c->table[s].push_back(page);
+        }
+    }
+    return KVCAR_OK;
+}
+
+// bring the device copies of the page table and sequence lengths up to date, in stream order
+kvcar_status flush_tables(kvcar_ctx *c, cudaStream_t st) {
+    if (c->pending.empty()) return KVCAR_OK;
+    int32_t *bt = reinterpret_cast<int32_t *>(c->ws + c->bt_off);
+    int32_t *ln = reinterpret_cast<int32_t *>(c->ws + c->len_off);
+    if (c->pending.size() > 4 * 240) {
+        // many changes: re-send both tables whole (pageable source: staged before the call returns)
+        const int mp = c->cfg.max_pages_per_seq;
+        std::vector<int32_t> full((size_t)c->cfg.max_seqs * mp, 0);
+        for (int s = 0; s < c->cfg.max_seqs; ++s)
+            for (size_t i = 0; i < c->table[s].size(); ++i) full[(size_t)s * mp + i] = c->table[s][i];
+        // the host mirror of the lengths is what the device must see once every pending update is applied
+        cudaError_t e = cudaMemcpyAsync(bt, full.data(), full.size() * 4, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ln, c->len.data(), c->len.size() * 4, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(c, e, "upload tables");
+        c->pending.clear();
+        return KVCAR_OK;
+    }
+    size_t done = 0;
+    while (done < c->pending.size()) {
+        TableUpdates u;
+        u.max_pages_per_seq = c->cfg.max_pages_per_seq;
+        u.n = (int)std::min<size_t>(240, c->pending.size() - done);
+        memcpy(u.e, c->pending.data() + done, (size_t)u.n * sizeof(int4));
+        cudaError_t e = launch_table_updates(bt, ln, u, st);
+        if (e != cudaSuccess) return cuda_fail(c, e, "table update launch");
+        ++c->launches;
+        done += u.n;
+    }
+    c->pending.clear();
+    return KVCAR_OK;
+}
+
+bool use_tensor_kernel(const kvcar_ctx *c) {
+    if (c->kernel == KVCAR_KERNEL_GENERIC) return false;
+    return c->tc.available;
+}
+
+}  // namespace
+
+// =============================================================================
+extern "C" {
+
+kvcar_status kvcar_create(const kvcar_config *cfg, kvcar_ctx **out_ctx) {
+    if (!cfg || !out_ctx) return KVCAR_ERR_INVALID_ARG;
+    const kvcar_config &g = *cfg;
+    if (g.n_layers <= 0 || g.n_q_heads <= 0 || g.n_kv_heads <= 0 || g.head_dim <= 0 || g.page_tokens <= 0 ||
+        g.max_seqs <= 0 || g.max_pages <= 0 || g.max_pages_per_seq <= 0)
+        return KVCAR_ERR_INVALID_ARG;
+    if (g.n_q_heads % g.n_kv_heads != 0 || g.n_kv_heads > KVCAR_MAX_KV_HEADS || g.n_q_heads > KVCAR_MAX_Q_HEADS ||
+        g.head_dim > KVCAR_MAX_HEAD_DIM || g.head_dim % 4 != 0)
+        return KVCAR_ERR_INVALID_ARG;
+    if (g.storage != KVCAR_F32 && g.storage != KVCAR_BF16) return KVCAR_ERR_INVALID_ARG;
+    kvcar_ctx *c = new (std::nothrow) kvcar_ctx();
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    c->cfg = g;
+    c->elem = g.storage == KVCAR_F32 ? 4 : 2;
+    for (int w = 0; w < 2; ++w) c->src[w].assign((size_t)g.n_layers * g.n_kv_heads, -1);
+    c->ae.resize((size_t)g.n_layers * 2);
+    c->free_pages.resize(g.max_pages);
+    for (int i = 0; i < g.max_pages; ++i) c->free_pages[i] = g.max_pages - 1 - i;  // back() pops 0 first
+    c->table.resize(g.max_seqs);
+    c->len.assign(g.max_seqs, 0);
+    c->open.assign(g.max_seqs, 0);
+    *out_ctx = c;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_destroy(kvcar_ctx *ctx) {
+    if (!ctx) return KVCAR_ERR_INVALID_ARG;
+    tc_destroy(ctx->tc);
+    delete ctx;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_set_reuse_map(kvcar_ctx *c, const int32_t *src_k, const int32_t *src_v) {
+    if (!c || !src_k || !src_v) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (c->bound) return fail(c, KVCAR_ERR_STATE, "reuse map is frozen after kvcar_bind_memory");
+    for (const AEHost &a : c->ae)
+        if (a.set) return fail(c, KVCAR_ERR_STATE, "set the reuse map before the autoencoders");
+    const int hkv = c->cfg.n_kv_heads, n = c->cfg.n_layers * hkv;
+    const int32_t *in[2] = {src_k, src_v};
+    for (int w = 0; w < 2; ++w)
+        for (int i = 0; i < n; ++i) {
+            int v = in[w][i];
+            if (v < -1 || v >= hkv) return fail(c, KVCAR_ERR_INVALID_ARG, "reuse entry out of range");
+            if (i < hkv && v != -1) return fail(c, KVCAR_ERR_INVALID_ARG, "layer 0 has no layer below it");
+        }
+    for (int w = 0; w < 2; ++w) c->src[w].assign(in[w], in[w] + n);
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_set_autoencoder(kvcar_ctx *c, int32_t layer, int32_t which, const kvcar_ae *ae) {
+    if (!c || !ae) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (c->bound) return fail(c, KVCAR_ERR_STATE, "autoencoders are frozen after kvcar_bind_memory");
+    if (layer < 0 || layer >= c->cfg.n_layers || (which != 0 && which != 1))
+        return fail(c, KVCAR_ERR_INVALID_ARG, "layer/which out of range");
+    const int n_stored = (int)stored_heads(c, layer, which).size();
+    if (ae->in_dim != n_stored * c->cfg.head_dim || ae->in_dim <= 0)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "in_dim must equal stored heads * head_dim");
+    if (ae->hidden <= 0 || ae->latent <= 0) return fail(c, KVCAR_ERR_INVALID_ARG, "non-positive width");
+    const float *ptrs[] = {ae->enc_w1, ae->enc_b1, ae->enc_bn, ae->enc_w2, ae->enc_b2,
+                           ae->dec_w1, ae->dec_b1, ae->dec_bn, ae->dec_w2, ae->dec_b2};
+    for (const float *p : ptrs)
+        if (!p) return fail(c, KVCAR_ERR_INVALID_ARG, "null weight pointer");
+    AEHost &a = c->ae[layer * 2 + which];
+    a.set = true;
+    a.in_dim = ae->in_dim;
+    a.hidden = ae->hidden;
+    a.latent = ae->latent;
+    a.slope = ae->leaky_slope;
+    a.eps = ae->bn_eps;
+    const size_t I = a.in_dim, M = a.hidden, D = a.latent;
+    a.enc_w1.assign(ae->enc_w1, ae->enc_w1 + M * I);
+    a.enc_b1.assign(ae->enc_b1, ae->enc_b1 + M);
+    a.enc_bn.assign(ae->enc_bn, ae->enc_bn + 4 * M);
+    a.enc_w2.assign(ae->enc_w2, ae->enc_w2 + D * M);
+    a.enc_b2.assign(ae->enc_b2, ae->enc_b2 + D);
+    a.dec_w1.assign(ae->dec_w1, ae->dec_w1 + M * D);
+    a.dec_b1.assign(ae->dec_b1, ae->dec_b1 + M);
+    a.dec_bn.assign(ae->dec_bn, ae->dec_bn + 4 * M);
+    a.dec_w2.assign(ae->dec_w2, ae->dec_w2 + I * M);
+    a.dec_b2.assign(ae->dec_b2, ae->dec_b2 + I);
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_required_bytes(kvcar_ctx *c, size_t *pool, size_t *weights, size_t *workspace) {
+    if (!c || !pool || !weights || !workspace) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (!c->bound) compute_layout(c);
+    *pool = c->pool_bytes;
+    *weights = c->weights_bytes;
+    *workspace = c->ws_bytes;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void *weights, size_t weights_bytes,
+                               void *workspace, size_t workspace_bytes, void *stream) {
+    if (!c || !pool || !weights || !workspace) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (c->bound) return fail(c, KVCAR_ERR_STATE, "memory already bound");
+    if (((uintptr_t)pool | (uintptr_t)weights | (uintptr_t)workspace) & 255)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "buffers must be 256-byte aligned");
+    compute_layout(c);
+    if (pool_bytes < c->pool_bytes || weights_bytes < c->weights_bytes || workspace_bytes < c->ws_bytes)
+        return fail(c, KVCAR_ERR_WORKSPACE, "a bound buffer is smaller than kvcar_required_bytes reports");
+    cudaStream_t st = (cudaStream_t)stream;
+    const kvcar_config &g = c->cfg;
+    const int nl = g.n_layers, hkv = g.n_kv_heads, hd = g.head_dim;
+    c->pool = (char *)pool;
+    c->weights = (char *)weights;
+    c->ws = (char *)workspace;
+
+    std::vector<char> img(c->weights_bytes, 0);
+    struct Packed {
+        size_t enc_w1t, enc_w2t, dec_w1t, dec_w2t, enc_s, enc_t, enc_b2, dec_s, dec_t, dec_b2, w1k, w2k;
+    };
+    std::vector<Packed> pk(nl * 2);
+    size_t w = 0;
+    for (int i = 0; i < nl * 2; ++i) {
+        const AEHost &a = c->ae[i];
+        if (!a.set) continue;
+        const size_t I = a.in_dim, M = a.hidden, D = a.latent, E = c->elem;
+        Packed &p = pk[i];
+        p.enc_w1t = w;
+        p.enc_w2t = p.enc_w1t + I * M * E;
+        p.dec_w1t = p.enc_w2t + M * D * E;
+        p.dec_w2t = p.dec_w1t + D * M * E;
+        w = align_up(w + 2 * (I * M + M * D) * E, 256);
+        p.enc_s = w;
+        p.enc_t = p.enc_s + M * 4;
+        p.dec_s = p.enc_t + M * 4;
+        p.dec_t = p.dec_s + M * 4;
+        p.enc_b2 = p.dec_t + M * 4;
+        p.dec_b2 = p.enc_b2 + D * 4;
+        w = align_up(w + (4 * M + D + I) * 4, 256);
+        put_transposed(&img[p.enc_w1t], a.enc_w1.data(), (int)M, (int)I, g.storage);  // [M][I] -> [I][M]
+        put_transposed(&img[p.enc_w2t], a.enc_w2.data(), (int)D, (int)M, g.storage);  // [D][M] -> [M][D]
+        put_transposed(&img[p.dec_w1t], a.dec_w1.data(), (int)M, (int)D, g.storage);  // [M][D] -> [D][M]
+        put_transposed(&img[p.dec_w2t], a.dec_w2.data(), (int)I, (int)M, g.storage);  // [I][M] -> [M][I]
+        fuse_bn(a.enc_b1, a.enc_bn, (int)M, a.eps, (float *)&img[p.enc_s], (float *)&img[p.enc_t]);
+        fuse_bn(a.dec_b1, a.dec_bn, (int)M, a.eps, (float *)&img[p.dec_s], (float *)&img[p.dec_t]);
+        memcpy(&img[p.enc_b2], a.enc_b2.data(), D * 4);
+        memcpy(&img[p.dec_b2], a.dec_b2.data(), I * 4);
+        if (g.storage == KVCAR_BF16) {
+            p.w1k = w;
+            p.w2k = p.w1k + M * D * 2;
+            w = align_up(w + (M * D + I * M) * 2, 256);
+            put_elems(&img[p.w1k], a.dec_w1.data(), M * D, KVCAR_BF16);
+            put_elems(&img[p.w2k], a.dec_w2.data(), I * M, KVCAR_BF16);
+        }
+    }
+
+    // per-layer decode plans
+    c->plans_host.assign(nl, LayerPlan{});
+    LayerPlan *plans = c->plans_host.data();
+    for (int l = 0; l < nl; ++l) {
+        LayerPlan &lp = plans[l];
+        memset(&lp, 0, sizeof(lp));
+        for (int which = 0; which < 2; ++which) {
+            WhichPlan &wp = lp.w[which];
+            wp.n_src = 0;
+            for (int h = 0; h < hkv; ++h) {
+                Resolved r = resolve(c, l, h, which);
+                lp.cur[which][h] = c->pool + c->cur_off[r.root_layer * 2 + which];
+                lp.cur_head[which][h] = r.root_head;
+                int s = 0;
+                for (; s < wp.n_src; ++s)
+                    if (wp.src[s].src_layer == r.root_layer) break;
+                if (s == wp.n_src) {
+                    SourcePlan &sp = wp.src[wp.n_src++];
+                    const int idx = r.root_layer * 2 + which;
+                    const AEHost &a = c->ae[idx];
+                    sp.src_layer = r.root_layer;
+                    sp.pool = c->pool + c->pool_off[idx];
+                    sp.width = c->width[idx];
+                    sp.compressed = a.set ? 1 : 0;
+                    sp.n_need = 0;
+                    if (a.set) {
+                        sp.d = a.latent;
+                        sp.m = a.hidden;
+                        sp.in_dim = a.in_dim;
+                        sp.slope = a.slope;
+                        sp.w1t = c->weights + pk[idx].dec_w1t;
+                        sp.w2t = c->weights + pk[idx].dec_w2t;
+                        sp.s1 = (const float *)(c->weights + pk[idx].dec_s);
+                        sp.t1 = (const float *)(c->weights + pk[idx].dec_t);
+                        sp.b2 = (const float *)(c->weights + pk[idx].dec_b2);
+                        if (g.storage == KVCAR_BF16) {
+                            sp.w1k = c->weights + pk[idx].w1k;
+                            sp.w2k = c->weights + pk[idx].w2k;
+                        }
+                    } else {
+                        sp.d = sp.in_dim = sp.width;
+                        sp.m = 0;
+                    }
+                }
+                SourcePlan &sp = wp.src[s];
+                sp.kv_head[sp.n_need] = (int8_t)h;
+                sp.slot[sp.n_need] = (int8_t)r.slot;
+                ++sp.n_need;
+            }
+        }
+    }
+    memcpy(&img[c->plan_off], plans, (size_t)nl * sizeof(LayerPlan));
+
+    std::vector<EncPlan> enc(nl * 2);
+    for (int i = 0; i < nl * 2; ++i) {
+        EncPlan &e = enc[i];
+        memset(&e, 0, sizeof(e));
+        const AEHost &a = c->ae[i];
+        std::vector<int> heads = stored_heads(c, i / 2, i % 2);
+        e.pool = c->pool + c->pool_off[i];
+        e.cur = c->pool + c->cur_off[i];
+        e.width = c->width[i];
+        e.n_stored = (int)heads.size();
+        for (size_t k = 0; k < heads.size(); ++k) e.heads[k] = (int8_t)heads[k];
+        e.in_dim = e.n_stored * hd;
+        e.compressed = a.set ? 1 : 0;
+        if (a.set) {
+            e.d = a.latent;
+            e.m = a.hidden;
+            e.slope = a.slope;
+            e.w1t = c->weights + pk[i].enc_w1t;
+            e.w2t = c->weights + pk[i].enc_w2t;
+            e.s1 = (const float *)(c->weights + pk[i].enc_s);
+            e.t1 = (const float *)(c->weights + pk[i].enc_t);
+            e.b2 = (const float *)(c->weights + pk[i].enc_b2);
+        } else {
+            e.d = e.in_dim;
+        }
+    }
+    memcpy(&img[c->enc_off], enc.data(), enc.size() * sizeof(EncPlan));
+
+    cudaError_t e = cudaMemcpyAsync(c->weights, img.data(), img.size(), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->part_off, st);  // tables, lengths, status
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "upload of packed weights");
+    c->bound = true;
+    c->pending.clear();
+    // re-queue what host bookkeeping already holds (sequences opened / pages reserved before binding)
+    for (int s = 0; s < g.max_seqs; ++s) {
+        for (size_t i = 0; i < c->table[s].size(); ++i) c->pending.push_back(make_int4(0, s, (int)i, c->table[s][i]));
+        if (c->len[s]) c->pending.push_back(make_int4(1, s, 0, c->len[s]));
+    }
+    tc_setup(c->tc, c->cfg, plans, nl, (const LayerPlan *)(c->weights + c->plan_off), (size_t)g.max_pages * g.page_tokens);
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_set_kernel(kvcar_ctx *c, int32_t kernel) {
+    if (!c || kernel < 0 || kernel > 2) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown kernel family");
+    if (kernel == KVCAR_KERNEL_TENSOR && c->bound && !c->tc.available)
+        return fail(c, KVCAR_ERR_UNSUPPORTED, std::string("tensor-core kernel unavailable: ") + c->tc.why);
+    c->kernel = kernel;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_seq_open(kvcar_ctx *c, int32_t seq) {
+    if (!c || seq < 0 || seq >= c->cfg.max_seqs) return fail(c, KVCAR_ERR_INVALID_ARG, "sequence id out of range");
+    if (c->open[seq]) return fail(c, KVCAR_ERR_STATE, "sequence already open");
+    c->open[seq] = 1;
+    c->len[seq] = 0;
+    c->pending.push_back(make_int4(1, seq, 0, 0));
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_seq_close(kvcar_ctx *c, int32_t seq) {
+    if (!c || seq < 0 || seq >= c->cfg.max_seqs) return fail(c, KVCAR_ERR_INVALID_ARG, "sequence id out of range");
+    if (!c->open[seq]) return fail(c, KVCAR_ERR_STATE, "sequence not open");
+    for (int32_t p : c->table[seq]) c->free_pages.push_back(p);
+    c->table[seq].clear();
+    c->open[seq] = 0;
+    c->len[seq] = 0;
+    c->pending.push_back(make_int4(1, seq, 0, 0));
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_reserve(kvcar_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!check_seqs(c, seqs, n_seqs) || n_tokens <= 0) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    return reserve_pages(c, seqs, n_seqs, n_tokens);
+}
+
+kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens,
+                                 const void *k, const void *v, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (layer < 0 || layer >= c->cfg.n_layers || !k || !v || n_tokens <= 0)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer, pointer or token count");
+    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "k/v must be 16-byte aligned");
+    kvcar_status s = reserve_pages(c, seqs, n_seqs, n_tokens);
+    if (s != KVCAR_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    s = flush_tables(c, st);
+    if (s != KVCAR_OK) return s;
+    EncodeArgs a{};
+    a.plan = reinterpret_cast<const EncPlan *>(c->weights + c->enc_off) + layer * 2;
+    a.block_table = reinterpret_cast<const int32_t *>(c->ws + c->bt_off);
+    a.seq_len = reinterpret_cast<const int32_t *>(c->ws + c->len_off);
+    a.k = k;
+    a.v = v;
+    a.max_pages_per_seq = c->cfg.max_pages_per_seq;
+    a.page_tokens = c->cfg.page_tokens;
+    a.n_tokens = n_tokens;
+    a.kv_width = c->cfg.n_kv_heads * c->cfg.head_dim;
+    a.hd = c->cfg.head_dim;
+    SeqList sl;
+    sl.n = n_seqs;
+    memcpy(sl.id, seqs, (size_t)n_seqs * 4);
+    cudaError_t e = launch_encode_generic(a, sl, c->cfg.storage, c->max_in, c->max_m, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "encode launch");
+    ++c->launches;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_advance(kvcar_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!check_seqs(c, seqs, n_seqs) || n_tokens <= 0) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    const int P = c->cfg.page_tokens;
+    for (int i = 0; i < n_seqs; ++i)
+        if (c->len[seqs[i]] + n_tokens > (int)c->table[seqs[i]].size() * P)
+            return fail(c, KVCAR_ERR_STATE, "advance beyond reserved pages");
+    for (int i = 0; i < n_seqs; ++i) {
+        c->len[seqs[i]] += n_tokens;
+        c->pending.push_back(make_int4(1, seqs[i], 0, c->len[seqs[i]]));
+    }
+    if (c->bound) return flush_tables(c, (cudaStream_t)stream);
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *q,
+                                    void *out, uint32_t flags, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (layer < 0 || layer >= c->cfg.n_layers || !q || !out)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
+    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    if (flags & ~KVCAR_INCLUDE_CURRENT_EXACT) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    cudaStream_t st = (cudaStream_t)stream;
+    kvcar_status s = flush_tables(c, st);
+    if (s != KVCAR_OK) return s;
+    const kvcar_config &g = c->cfg;
+    int max_len = 0;
+    for (int i = 0; i < n_seqs; ++i) max_len = std::max(max_len, c->len[seqs[i]]);
+    DecodeArgs a{};
+    a.plan = reinterpret_cast<const LayerPlan *>(c->weights + c->plan_off) + layer;
+    a.block_table = reinterpret_cast<const int32_t *>(c->ws + c->bt_off);
+    a.seq_len = reinterpret_cast<const int32_t *>(c->ws + c->len_off);
+    a.q = q;
+    a.out = out;
+    a.partials = reinterpret_cast<float *>(c->ws + c->part_off);
+    a.status = reinterpret_cast<int32_t *>(c->ws + c->status_off);
+    a.max_pages_per_seq = g.max_pages_per_seq;
+    a.page_tokens = g.page_tokens;
+    a.hq = g.n_q_heads;
+    a.hkv = g.n_kv_heads;
+    a.hd = g.head_dim;
+    a.chunk_tokens = c->chunk_tokens;
+    a.max_chunks = c->max_chunks;
+    a.flags = flags;
+    a.scale = 1.0f / std::sqrt((float)g.head_dim);
+    SeqList sl;
+    sl.n = n_seqs;
+    memcpy(sl.id, seqs, (size_t)n_seqs * 4);
+    const int n_chunks = (max_len + c->chunk_tokens - 1) / c->chunk_tokens;
+    if (n_chunks > 0) {
+        const bool want_tc = use_tensor_kernel(c) && tc_layer_supported(c->tc, layer);
+        if (c->kernel == KVCAR_KERNEL_TENSOR && !want_tc)
+            return fail(c, KVCAR_ERR_UNSUPPORTED, std::string("tensor-core kernel cannot run this layer: ") + c->tc.why);
+        cudaError_t e;
+        if (want_tc) {
+            e = tc_launch_decode(c->tc, a, sl, layer, n_chunks, st);
+        } else {
+            if (decode_generic_smem(a.hq, a.hd, c->max_d, c->max_m) > 227 * 1024)
+                return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");
+            e = launch_decode_generic(a, sl, g.storage, c->max_d, c->max_m, n_chunks, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(c, e, "decode launch");
+        ++c->launches;
+    }
+    cudaError_t e = launch_combine(a, sl, g.storage, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "combine launch");
+    ++c->launches;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_step_layer_host(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                   const void *k_host, const void *v_host, const void *q_host, void *out_host,
+                                   uint32_t flags, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (!k_host || !v_host || !q_host || !out_host) return fail(c, KVCAR_ERR_INVALID_ARG, "null host buffer");
+    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    const kvcar_config &g = c->cfg;
+    const size_t kvb = align_up((size_t)n_seqs * g.n_kv_heads * g.head_dim * c->elem, 256);
+    const size_t qb = align_up((size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, 256);
+    char *dk = c->ws + c->stage_off, *dv = dk + kvb, *dq = dv + kvb, *dout = dq + qb;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(dk, k_host, (size_t)n_seqs * g.n_kv_heads * g.head_dim * c->elem,
+                                    cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(dv, v_host, (size_t)n_seqs * g.n_kv_heads * g.head_dim * c->elem, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(dq, q_host, (size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "host to device copy");
+    kvcar_status s = kvcar_encode_append(c, layer, seqs, n_seqs, 1, dk, dv, stream);
+    if (s != KVCAR_OK) return s;
+    s = kvcar_decode_attention(c, layer, seqs, n_seqs, dq, dout, flags, stream);
+    if (s != KVCAR_OK) return s;
+    e = cudaMemcpyAsync(out_host, dout, (size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "device to host copy");
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_debug_resolve(kvcar_ctx *c, int32_t layer, int32_t kv_head, int32_t which, int32_t *root_layer,
+                                 int32_t *root_head, int32_t *slot) {
+    if (!c || !root_layer || !root_head || !slot) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (layer < 0 || layer >= c->cfg.n_layers || kv_head < 0 || kv_head >= c->cfg.n_kv_heads || (which & ~1))
+        return fail(c, KVCAR_ERR_INVALID_ARG, "index out of range");
+    Resolved r = resolve(c, layer, kv_head, which);
+    *root_layer = r.root_layer;
+    *root_head = r.root_head;
+    *slot = r.slot;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_debug_locate(kvcar_ctx *c, int32_t seq, int32_t token, int32_t *page, int64_t *row) {
+    if (!c || !page || !row) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (seq < 0 || seq >= c->cfg.max_seqs || !c->open[seq] || token < 0)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "sequence not open or token negative");
+    const int P = c->cfg.page_tokens;
+    if (token / P >= (int)c->table[seq].size()) return fail(c, KVCAR_ERR_INVALID_ARG, "token lies in no reserved page");
+    *page = c->table[seq][token / P];
+    *row = (int64_t)*page * P + token % P;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_seq_len(kvcar_ctx *c, int32_t seq, int32_t *len) {
+    if (!c || !len || seq < 0 || seq >= c->cfg.max_seqs || !c->open[seq])
+        return fail(c, KVCAR_ERR_INVALID_ARG, "sequence not open");
+    *len = c->len[seq];
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_pool_layout(kvcar_ctx *c, int32_t layer, int32_t which, size_t *offset, size_t *row_pitch,
+                               int32_t *width) {
+    if (!c || !offset || !row_pitch || !width) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (layer < 0 || layer >= c->cfg.n_layers || (which & ~1)) return fail(c, KVCAR_ERR_INVALID_ARG, "index out of range");
+    if (!c->bound) compute_layout(c);
+    const int i = layer * 2 + which;
+    *offset = c->pool_off[i];
+    *width = c->width[i];
+    *row_pitch = (size_t)c->width[i] * c->elem;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *c, double *compressed, double *uncompressed) {
+    if (!c || !compressed || !uncompressed) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    double comp = 0;
+    for (int i = 0; i < c->cfg.n_layers * 2; ++i) comp += (double)stored_width(c, i / 2, i % 2) * c->elem;
+    *compressed = comp;
+    *uncompressed = 2.0 * c->cfg.n_layers * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_layer_work_per_token(kvcar_ctx *c, int32_t layer, double *bytes, double *flops) {
+    if (!c || !bytes || !flops || layer < 0 || layer >= c->cfg.n_layers)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "bad argument");
+    const int hkv = c->cfg.n_kv_heads, hd = c->cfg.head_dim;
+    double b = 0, f = 0;
+    for (int which = 0; which < 2; ++which) {
+        std::vector<int> need(c->cfg.n_layers, 0);
+        for (int h = 0; h < hkv; ++h) ++need[resolve(c, layer, h, which).root_layer];
+        for (int s = 0; s < c->cfg.n_layers; ++s) {
+            if (!need[s]) continue;
+            const AEHost &a = c->ae[s * 2 + which];
+            b += (double)stored_width(c, s, which) * c->elem;
+            if (a.set) f += 2.0 * a.latent * a.hidden + 2.0 * a.hidden * hd * need[s];
+        }
+    }
+    f += 4.0 * c->cfg.n_q_heads * hd;  // q.K and p.V
+    *bytes = b;
+    *flops = f;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_launch_count(kvcar_ctx *c, int64_t *count) {
+    if (!c || !count) return KVCAR_ERR_INVALID_ARG;
+    *count = c->launches;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_sync_status(kvcar_ctx *c, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    if (c->bound) {
+        int32_t status = 0;
+        e = cudaMemcpy(&status, c->ws + c->status_off, 4, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return cuda_fail(c, e, "status read");
+        if (status != 0) {
+            cudaMemset(c->ws + c->status_off, 0, 4);
+            char buf[96];
+            snprintf(buf, sizeof buf, "device-side bounded wait ran out (code 0x%x)", status);
+            return fail(c, KVCAR_ERR_DEVICE_TIMEOUT, buf);
+        }
+    }
+    return KVCAR_OK;
+}
+
+const char *kvcar_last_error(kvcar_ctx *c) { return c ? c->err.c_str() : "null context"; }
+
+}  // extern "C"

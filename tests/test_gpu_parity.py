@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, on
+the same seeded inputs, through the C ABI.  Sizes are chosen so that the oracle
+finishes in seconds while the kernels still see several tiles, several pages and
+ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import kvcar_synth as synth
+from kvcar_harness import Pair, assert_close
+from oracle.kvcar_oracle import K, V
+from paper_2512_06727_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [B.KERNEL_GENERIC, B.KERNEL_AUTO]
+KNAME = {B.KERNEL_GENERIC: "generic", B.KERNEL_AUTO: "auto"}
+
+
+def _check_step(res, storage, what):
+    worst = 0.0
+    for l, (got, ref, rows) in res.items():
+        err, rel = assert_close(got[rows], ref, storage, f"{what} layer {l}")
+        worst = max(worst, err)
+    return worst
+
+
+def test_config1_fp32_single_layer():
+    """BASELINE config 1 exactly: one GPT-2-small-shaped layer, 768->384, batch 1,
+    128 cached tokens, one decode step, fp32, no reuse; max abs error <= 1e-4."""
+    w = synth.CONFIGS["c1"]
+    p = Pair(w, max_seqs=1, max_pages=4, max_pages_per_seq=4)
+    p.open([0])
+    p.prefill([0], w.cached_tokens)
+    p.check_latents([0])
+    res = p.decode_step([0], 0)
+    got, ref, rows = res[0]
+    err, rel = assert_close(got[rows], ref, "f32", "config 1")
+    assert err <= 1e-4
+    assert p.s.ctx.cache_bytes_per_token() == (2 * 384 * 4, 2 * 768 * 4)
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_gpt2_shape_stack_bf16_with_reuse(kernel):
+    """Config-2-shaped stack (12 layers x 12 heads, latent 32/head, 25 % reuse),
+    reduced batch and ragged lengths, two decode steps with encode-append."""
+    w = synth.scaled(synth.CONFIGS["c2"], batch=3, cached_tokens=0, decode_steps=2)
+    p = Pair(w, max_seqs=4, max_pages=16, max_pages_per_seq=5, kernel=kernel)
+    seqs = [2, 0, 3]
+    p.open(seqs)
+    p.prefill([2], 200)
+    p.prefill([0], 131)
+    p.prefill([3], 64)
+    p.check_latents(seqs)
+    for step in range(2):
+        _check_step(p.decode_step(seqs, step), "bf16", f"step {step}")
+    p.check_latents(seqs)
+    assert p.s.ctx.cache_bytes_per_token() == p.o.cache_bytes_per_token()
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_tinyllama_shape_gqa_stack_bf16_with_reuse(kernel):
+    """Config-3-shaped GQA stack (22 layers, 32 query / 4 KV heads, latent 32/head,
+    20 % reuse), K and V reuse maps different, ragged lengths incl. 1 token."""
+    w = synth.scaled(synth.CONFIGS["c3"], batch=4, cached_tokens=0, decode_steps=2)
+    src_k = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    src_v = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed + 7)
+    p = Pair(w, max_seqs=4, max_pages=20, max_pages_per_seq=6, src_k=src_k, src_v=src_v, kernel=kernel)
+    seqs = [0, 1, 2, 3]
+    p.open(seqs)
+    for s, n in zip(seqs, (300, 257, 128, 1)):
+        p.prefill([s], n)
+    p.check_latents(seqs)
+    for step in range(2):
+        _check_step(p.decode_step(seqs, step), "bf16", f"step {step}")
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_peaked_softmax_and_planted_key(kernel):
+    """N(0,1) inputs give near-uniform softmax, under which a token-indexing bug
+    hardly moves the output: repeat with queries scaled x8 and with one cached key
+    made proportional to the query."""
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, batch=2, cached_tokens=0, decode_steps=1, reuse_frac=0.34)
+    p = Pair(w, max_seqs=2, max_pages=12, max_pages_per_seq=6, kernel=kernel)
+    seqs = [0, 1]
+    p.open(seqs)
+    p.prefill(seqs, 333)
+    res = p.decode_step(seqs, 0, q_scale=8.0)
+    _check_step(res, "bf16", "q x8")
+    # the softmax really is peaked: the largest probability of some head exceeds 0.5
+    out, probs = p.o.decode_attention(2, [0], np.stack([synth.make_q(w, 2, 0, 0, scale=8.0)]),
+                                      include_current=False, return_probs=True)
+    assert max(float(pr.max()) for pr in probs) > 0.5
+    # planted key: make token 77's pre-compression K of every head a multiple of one query head, raw layer 0
+    w2 = synth.scaled(w, n_layers=1, reuse_frac=0.0)
+    p2 = Pair(w2, max_seqs=1, max_pages=4, max_pages_per_seq=4, compress=False, kernel=kernel)
+    p2.open([0])
+    q = synth.make_q(w2, 0, 0, 0)
+    k = synth.make_kv(w2, 0, K, 0, 0, 150)[None].copy()
+    v = synth.make_kv(w2, 0, V, 0, 0, 150)[None].copy()
+    for g in range(w2.n_kv_heads):
+        k[0, 77, g * 64:(g + 1) * 64] = synth.to_bf16_grid(6.0 * q[g * 8])
+    p2.append(0, [0], k, v)
+    p2.advance([0], 150)
+    got, ref, rows = p2.attention(0, [0], q[None], include_current=False)
+    assert_close(got, ref, "bf16", "planted key")
+    for g in range(w2.n_kv_heads):   # head g*8 attends almost only to token 77
+        assert np.max(np.abs(got[0, g * 8] - v[0, 77, g * 64:(g + 1) * 64])) < 0.05
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_edge_cases_empty_current_only_and_single_token(kernel):
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=3, reuse_frac=0.5)
+    p = Pair(w, max_seqs=3, max_pages=8, max_pages_per_seq=3, kernel=kernel)
+    seqs = [0, 1, 2]
+    p.open(seqs)
+    p.prefill([1], 1)
+    p.prefill([2], 65)
+    # seq 0 has nothing cached: with the current token the output is that token's exact V
+    res = p.decode_step(seqs, 0)
+    _check_step(res, "bf16", "current only")
+    # nothing cached and no current token: zeros
+    p3 = Pair(w, max_seqs=1, max_pages=2, max_pages_per_seq=2, kernel=kernel)
+    p3.open([0])
+    got, ref, rows = p3.attention(0, [0], synth.make_q(w, 0, 0, 0)[None], include_current=False)
+    assert np.all(got == 0) and np.all(ref == 0)
+    # cached tokens only (current token attended through its latent after advance)
+    got, ref, rows = p.attention(1, seqs, np.stack([synth.make_q(w, 1, s, 9) for s in seqs]), include_current=False)
+    assert_close(got, ref, "bf16", "cached only")
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_uncompressed_twin_and_mixed_stack(kernel):
+    """No autoencoders (raw K/V pages, reuse still redirects heads) and a stack
+    with autoencoders in some layers only (Table 2's "N layers" rows)."""
+    w = synth.scaled(synth.CONFIGS["c2"], n_layers=4, batch=2, reuse_frac=0.3)
+    for layers, compress in ((None, False), ([1, 2], True)):
+        p = Pair(w, max_seqs=2, max_pages=8, max_pages_per_seq=4, compressed_layers=layers, compress=compress,
+                 kernel=kernel)
+        p.open([0, 1])
+        p.prefill([0], 190)
+        p.prefill([1], 70)
+        p.check_latents([0, 1])
+        _check_step(p.decode_step([0, 1], 0), "bf16", f"layers={layers}")
+        assert p.s.ctx.cache_bytes_per_token() == p.o.cache_bytes_per_token()
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_physical_page_permutation_is_bit_invariant(kernel):
+    """The same logical cache laid out on different physical pages must give
+    bit-identical outputs."""
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=1, reuse_frac=0.25)
+
+    def run(scramble):
+        p = Pair(w, max_seqs=3, max_pages=12, max_pages_per_seq=6, kernel=kernel, with_oracle=False)
+        if scramble:
+            p.open([1, 2])
+            p.s.ctx.reserve([1], 130); p.s.ctx.reserve([2], 70)
+            p.s.ctx.seq_close(1); p.s.ctx.seq_close(2)
+        p.open([0])
+        p.prefill([0], 200)
+        pages = [p.s.ctx.debug_locate(0, t)[0] for t in range(0, 200, 64)]
+        res = p.decode_step([0], 0)
+        return pages, {l: r[0] for l, r in res.items()}
+    pa, a = run(False)
+    pb, b = run(True)
+    assert pa != pb
+    for l in a:
+        assert np.array_equal(a[l], b[l])
+
+
+def test_fp32_stack_with_reuse_generic():
+    """fp32 mode on a multi-layer stack with chains of reuse; 1e-4 absolute."""
+    w = synth.scaled(synth.CONFIGS["c2"], n_layers=4, batch=2, storage="f32", reuse_frac=0.5)
+    p = Pair(w, max_seqs=2, max_pages=8, max_pages_per_seq=4)
+    p.open([0, 1])
+    p.prefill([0], 150)
+    p.prefill([1], 33)
+    p.check_latents([0, 1])
+    for step in range(2):
+        _check_step(p.decode_step([0, 1], step), "f32", f"step {step}")
+
+
+def test_host_buffer_entry_point_matches_device_entry_points():
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=2, reuse_frac=0.25)
+    p = Pair(w, max_seqs=2, max_pages=8, max_pages_per_seq=4)
+    seqs = [0, 1]
+    p.open(seqs)
+    p.prefill(seqs, 100)
+    dt = p.s.dtype
+    for l in range(w.n_layers):
+        k = np.stack([synth.make_kv(w, l, K, s, 100, 1) for s in seqs])
+        v = np.stack([synth.make_kv(w, l, V, s, 100, 1) for s in seqs])
+        q = np.stack([synth.make_q(w, l, s, 0) for s in seqs])
+        hk = torch.from_numpy(k).to(dt).pin_memory(); hv = torch.from_numpy(v).to(dt).pin_memory()
+        hq = torch.from_numpy(q).to(dt).pin_memory()
+        ho = torch.empty_like(hq).pin_memory()
+        p.s.ctx.step_layer_host(l, seqs, hk.data_ptr(), hv.data_ptr(), hq.data_ptr(), ho.data_ptr(),
+                                B.INCLUDE_CURRENT_EXACT, p.s.stream())
+        p.s.ctx.sync_status(p.s.stream())
+        p.o.encode_append(l, seqs, 1, k, v)
+        ref = p.o.decode_attention(l, seqs, q)
+        assert_close(ho.float().numpy().astype(np.float64), ref, "bf16", f"host entry layer {l}")
+
+
+def test_errors_leave_state_untouched():
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=1, batch=1, reuse_frac=0.0)
+    p = Pair(w, max_seqs=2, max_pages=2, max_pages_per_seq=2, with_oracle=False)
+    p.open([0, 1])
+    p.prefill([0], 64)
+    big = torch.zeros(1, 100, w.kv_width, dtype=p.s.dtype, device="cuda")
+    with pytest.raises(B.KvcarError) as e:      # 100 more tokens need 2 pages, 1 is left
+        p.s.ctx.encode_append(0, [0], 100, big.data_ptr(), big.data_ptr(), p.s.stream())
+    assert e.value.status == 3
+    assert p.s.ctx.seq_len(0) == 64
+    p.s.ctx.reserve([1], 64)                    # the last page is still available
+    with pytest.raises(B.KvcarError) as e:
+        p.s.ctx.decode_attention(0, [5], big.data_ptr(), big.data_ptr(), 0, p.s.stream())
+    assert e.value.status == 1

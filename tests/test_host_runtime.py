@@ -1,0 +1,167 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every declared symbol,
+and its integer bookkeeping (reuse resolution, page allocation, accounting)
+matches the oracle bit for bit.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import kvcar_synth as synth
+from oracle.kvcar_oracle import K, V, KVCAROracle
+from paper_2512_06727_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "kvcar.h")).read()
+    declared = sorted(set(re.findall(r"\b(kvcar_[a-z_0-9]+)\s*\(", header)))
+    assert len(declared) >= 20
+    lib = B.load()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert sorted(B.EXPORTS) == declared
+
+
+def _pair(w, src_k, src_v, max_seqs=6, max_pages=40, mpps=12, compressed_layers=None):
+    o = KVCAROracle(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, max_seqs, max_pages, w.storage)
+    c = B.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, max_seqs, max_pages, mpps,
+                  B.BF16 if w.storage == "bf16" else B.F32)
+    o.set_reuse_map(src_k, src_v)
+    c.set_reuse_map(src_k, src_v)
+    aes = synth.make_stack_autoencoders(w, src_k, src_v, layers=compressed_layers)
+    for (l, which), ae in aes.items():
+        o.set_autoencoder(l, which, ae)
+        c.set_autoencoder(l, which, ae)
+    return o, c
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_resolve_matches_oracle_on_benchmark_maps(name):
+    w = synth.CONFIGS[name]
+    src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    src_v = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed + 100)  # K and V differ
+    o, c = _pair(w, src, src_v)
+    for l in range(w.n_layers):
+        for h in range(w.n_kv_heads):
+            for which in (K, V):
+                assert c.debug_resolve(l, h, which) == o.resolve(l, h, which)
+    assert c.cache_bytes_per_token() == o.cache_bytes_per_token()
+
+
+def test_resolve_random_chains():
+    rng = np.random.default_rng(0)
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=9, n_kv_heads=4, n_q_heads=8)
+    for trial in range(20):
+        src_k = -np.ones((9, 4), np.int32)
+        src_v = -np.ones((9, 4), np.int32)
+        for s in (src_k, src_v):
+            mask = rng.random((8, 4)) < 0.6
+            s[1:][mask] = rng.integers(0, 4, size=int(mask.sum()))   # arbitrary head of the layer below
+        o = KVCAROracle(9, 8, 4, 64, 64, 1, 1)
+        c = B.Context(9, 8, 4, 64, 64, 1, 1, 1, B.F32)
+        o.set_reuse_map(src_k.reshape(-1), src_v.reshape(-1))
+        c.set_reuse_map(src_k.reshape(-1), src_v.reshape(-1))
+        for l in range(9):
+            for h in range(4):
+                for which in (K, V):
+                    assert c.debug_resolve(l, h, which) == o.resolve(l, h, which)
+
+
+def test_reuse_map_validation():
+    c = B.Context(3, 4, 2, 64, 64, 1, 1, 1, B.F32)
+    with pytest.raises(B.KvcarError) as e:
+        c.set_reuse_map([0, -1, -1, -1, -1, -1], [-1] * 6)
+    assert e.value.status == 1
+    with pytest.raises(B.KvcarError):
+        c.set_reuse_map([-1, -1, 2, -1, -1, -1], [-1] * 6)
+    with pytest.raises(B.KvcarError):
+        c.set_reuse_map([-1, -1, -2, -1, -1, -1], [-1] * 6)
+    c.set_reuse_map([-1, -1, 1, 0, 1, 1], [-1] * 6)
+    ae = synth.make_autoencoder(128, 96, 64, 0, 0, 0)
+    c.set_autoencoder(0, 0, ae)
+    with pytest.raises(B.KvcarError) as e:      # layer 2 stores no K head at all: in_dim 128 is wrong
+        c.set_autoencoder(2, 0, ae)
+    assert e.value.status == 1
+    with pytest.raises(B.KvcarError) as e:      # map is frozen once an autoencoder depends on it
+        c.set_reuse_map([-1] * 6, [-1] * 6)
+    assert e.value.status == 2
+
+
+def test_page_allocator_matches_oracle():
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, page_tokens=16)
+    src = np.full(2 * w.n_kv_heads, -1, np.int32)
+    o, c = _pair(w, src, src, max_seqs=6, max_pages=40, mpps=12)
+    rng = np.random.default_rng(1)
+    open_seqs = []
+    for step in range(400):
+        r = rng.random()
+        if r < 0.15 and len(open_seqs) < 6:
+            s = int(rng.choice([i for i in range(6) if i not in open_seqs]))
+            o.seq_open(s); c.seq_open(s); open_seqs.append(s)
+        elif r < 0.25 and open_seqs:
+            s = open_seqs.pop(int(rng.integers(len(open_seqs))))
+            o.seq_close(s); c.seq_close(s)
+        elif open_seqs:
+            k = int(rng.integers(1, len(open_seqs) + 1))
+            seqs = [int(x) for x in rng.permutation(open_seqs)[:k]]
+            n = int(rng.integers(1, 40))
+            if any(o.seq_len[s] + n > 12 * 16 for s in seqs):
+                with pytest.raises(B.KvcarError) as e:      # longer than max_pages_per_seq allows
+                    c.reserve(seqs, n)
+                assert e.value.status == 3
+                continue
+            try:
+                o.reserve(seqs, n)
+            except MemoryError:
+                with pytest.raises(B.KvcarError) as e:      # pool exhausted: refused, nothing taken
+                    c.reserve(seqs, n)
+                assert e.value.status == 3
+                continue
+            c.reserve(seqs, n)
+            o.advance(seqs, n); c.advance(seqs, n)
+        for s in open_seqs:
+            assert c.seq_len(s) == o.seq_len[s]
+            for t in range(0, o.seq_len[s], 7):
+                assert c.debug_locate(s, t) == o.locate(s, t)
+            if o.seq_len[s]:
+                assert c.debug_locate(s, o.seq_len[s] - 1) == o.locate(s, o.seq_len[s] - 1)
+
+
+def test_accounting_and_layout():
+    w = synth.CONFIGS["c2"]
+    src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    o, c = _pair(w, src, src, compressed_layers=list(range(10)))
+    assert c.cache_bytes_per_token() == o.cache_bytes_per_token()
+    pool_b, w_b, ws_b = c.required_bytes()
+    rows = 40 * 64
+    total = 0
+    last_end = 0
+    for l in range(w.n_layers):
+        for which in (K, V):
+            off, pitch, width = c.pool_layout(l, which)
+            assert width == o.stored_width(l, which) and pitch == width * 2
+            assert off % 256 == 0 and off >= last_end
+            last_end = off + rows * pitch
+            total += rows * pitch
+    assert pool_b >= total
+    # work model: no reuse, GPT-2-small shape -> 1536 latent bytes and 2 654 208 + 3072 flops per token-layer
+    w1 = synth.CONFIGS["c1"]
+    none = np.full(w1.n_kv_heads, -1, np.int32)
+    o1, c1 = _pair(synth.scaled(w1, storage="bf16"), none, none)
+    assert c1.layer_work_per_token(0) == (1536.0, 2654208.0 + 3072.0)
+
+
+def test_launching_calls_need_bound_memory():
+    c = B.Context(1, 4, 2, 64, 64, 2, 4, 2, B.BF16)
+    c.seq_open(0)
+    with pytest.raises(B.KvcarError) as e:
+        c.encode_append(0, [0], 1, 256, 256)
+    assert e.value.status == 2
+    with pytest.raises(B.KvcarError) as e:
+        c.decode_attention(0, [0], 256, 256)
+    assert e.value.status == 2
+    with pytest.raises(B.KvcarError):
+        B.Context(1, 5, 2, 64, 64, 2, 4, 2, B.BF16)      # query heads not a multiple of KV heads
