@@ -1,0 +1,491 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-CAR decode hot path on B200.
+
+One "step" = one decode step of the whole stack: for every layer, encoder +
+append of the new token's K/V, then decoder + attention over the latent cache
+(cached tokens restored, current token exact); then the sequence lengths advance.
+Metric: decode tokens/s (sequences x steps / time), whole job.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--batch B]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+Inputs are seeded and synthetic (N(0,1) K/V/Q, Xavier-uniform autoencoders, seeded
+reuse map) with the shapes of the paper's GPT-2 and TinyLLaMA workloads.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import kvcar_synth as synth  # noqa: E402
+
+METRIC = "decode tokens/s over latent KV cache"
+UNIT = "tokens/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--batch", type=int, default=None, help="override the batch (config 5 sweep)")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tensor"])
+    ap.add_argument("--uncompressed", action="store_true", help="raw K/V pages (the uncompressed twin)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle sample")
+    return ap.parse_args()
+
+
+def workload_of(args) -> synth.Workload:
+    w = synth.CONFIGS[args.workload]
+    if args.batch:
+        w = synth.with_batch(w, args.batch)
+    return w
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------
+def build_session(w: synth.Workload, args, torch, extra_steps: int):
+    from paper_2512_06727_b200 import binding as B
+    from paper_2512_06727_b200.session import Session
+    src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    aes = {} if args.uncompressed else synth.make_stack_autoencoders(w, src, src)
+    total = w.cached_tokens + extra_steps
+    pps = (total + w.page_tokens - 1) // w.page_tokens
+    kernel = {"auto": B.KERNEL_AUTO, "generic": B.KERNEL_GENERIC, "tensor": B.KERNEL_TENSOR}[args.kernel]
+    s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, w.batch, w.batch * pps, pps,
+                w.storage, src, src, aes, kernel=kernel)
+    return s, src, aes
+
+
+def prefill(sess, w, torch, keep_seqs=()):
+    """Fill the cache with w.cached_tokens tokens per sequence from the seeded
+    device generator; returns the raw rows of `keep_seqs` (host, for the oracle)."""
+    seqs = list(range(w.batch))
+    for q in seqs:
+        sess.ctx.seq_open(q)
+    g = torch.Generator(device=sess.device)
+    g.manual_seed(w.seed)
+    kept = {}
+    chunk = max(64, min(w.cached_tokens, (1 << 28) // max(1, w.batch * w.kv_width)))  # <= 256 Mi elements per tensor
+    chunk = (chunk // w.page_tokens) * w.page_tokens or w.page_tokens
+    t = 0
+    while t < w.cached_tokens:
+        n = min(chunk, w.cached_tokens - t)
+        for l in range(w.n_layers):
+            k = torch.randn(w.batch, n, w.kv_width, generator=g, device=sess.device, dtype=torch.float32).to(sess.dtype)
+            v = torch.randn(w.batch, n, w.kv_width, generator=g, device=sess.device, dtype=torch.float32).to(sess.dtype)
+            sess.ctx.encode_append(l, seqs, n, k.data_ptr(), v.data_ptr(), sess.stream())
+            for q in keep_seqs:
+                kept.setdefault((l, q), []).append((k[q].float().cpu().numpy(), v[q].float().cpu().numpy()))
+            torch.cuda.current_stream().synchronize()
+        sess.ctx.advance(seqs, n, sess.stream())
+        t += n
+    sess.ctx.sync_status(sess.stream())
+    return kept
+
+
+def step_inputs(sess, w, torch, n_steps):
+    g = torch.Generator(device=sess.device)
+    g.manual_seed(w.seed + 1000)
+    k = torch.randn(n_steps, w.n_layers, w.batch, w.kv_width, generator=g, device=sess.device).to(sess.dtype)
+    v = torch.randn(n_steps, w.n_layers, w.batch, w.kv_width, generator=g, device=sess.device).to(sess.dtype)
+    q = torch.randn(n_steps, w.n_layers, w.batch, w.n_q_heads, w.head_dim, generator=g, device=sess.device).to(sess.dtype)
+    out = torch.empty_like(q)
+    return k, v, q, out
+
+
+def run_step(sess, w, seqs, k, v, q, out, i, stream, flags):
+    ctx = sess.ctx
+    for l in range(w.n_layers):
+        ctx.encode_append(l, seqs, 1, k[i, l].data_ptr(), v[i, l].data_ptr(), stream)
+        ctx.decode_attention(l, seqs, q[i, l].data_ptr(), out[i, l].data_ptr(), flags, stream)
+    ctx.advance(seqs, 1, stream)
+
+
+def work_per_step(sess, w, cached_tokens):
+    """Algorithmic bytes / flops of the decode-attention kernels of one step."""
+    by = fl = 0.0
+    for l in range(w.n_layers):
+        b, f = sess.ctx.layer_work_per_token(l)
+        by += b * cached_tokens * w.batch
+        fl += f * cached_tokens * w.batch
+    return by, fl
+
+
+# ----------------------------------------------------------------------------
+def oracle_sample(w, src, aes, kept, steps_k, steps_v, steps_q, budget_s, gpu_out=None):
+    """Time the CPU oracle as it stands on (sequence, layer) pairs of this
+    workload.  Returns tokens/s scaled to the whole batch and stack, plus the
+    largest deviation of the GPU outputs on the sampled pairs (if given)."""
+    from oracle.kvcar_oracle import KVCAROracle
+    seqs = sorted({q for (_, q) in kept})
+    pps = (w.cached_tokens + 4 + w.page_tokens - 1) // w.page_tokens
+    o = KVCAROracle(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, max(seqs) + 1,
+                    len(seqs) * pps, w.storage)
+    o.set_reuse_map(src, src)
+    for (l, which), ae in aes.items():
+        o.set_autoencoder(l, which, ae)
+    for q in seqs:
+        o.seq_open(q)
+    # untimed: fill the oracle's own cache from the same raw rows
+    n_chunks = len(kept[(0, seqs[0])])
+    for c in range(n_chunks):
+        n = kept[(0, seqs[0])][c][0].shape[0]
+        for l in range(w.n_layers):
+            k = np.stack([kept[(l, q)][c][0] for q in seqs])
+            v = np.stack([kept[(l, q)][c][1] for q in seqs])
+            o.encode_append(l, seqs, n, k, v)
+        o.advance(seqs, n)
+    # timed: decode step 0 on the sampled pairs, stopping when the budget is spent
+    t0 = time.perf_counter()
+    pairs = 0
+    worst = 0.0
+    for q in seqs:
+        for l in range(w.n_layers):
+            o.encode_append(l, [q], 1, steps_k[l][q][None, None], steps_v[l][q][None, None])
+            ref = o.decode_attention(l, [q], steps_q[l][q][None])
+            pairs += 1
+            if gpu_out is not None:
+                worst = max(worst, float(np.max(np.abs(gpu_out[l][q] - ref[0]))))
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    per_pair = dt / pairs
+    step_time = per_pair * w.batch * w.n_layers
+    return {"value": w.batch / step_time, "pairs": pairs, "seconds": dt, "max_abs_err_vs_gpu": worst}
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+# ----------------------------------------------------------------------------
+def run_reference(args):
+    """The CPU oracle as the reference arm: each step is a bounded sample of
+    (sequence, layer) pairs of the workload, scaled to the whole batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workload_of(args)
+    src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    aes = synth.make_stack_autoencoders(w, src, src)
+    from oracle.kvcar_oracle import KVCAROracle
+    pps = (w.cached_tokens + args.steps + args.warmup + w.page_tokens) // w.page_tokens
+    o = KVCAROracle(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, 1, pps, w.storage)
+    o.set_reuse_map(src, src)
+    for (l, which), ae in aes.items():
+        o.set_autoencoder(l, which, ae)
+    o.seq_open(0)
+    rng = np.random.default_rng(w.seed)
+    blk = 1024
+    t = 0
+    while t < w.cached_tokens:
+        n = min(blk, w.cached_tokens - t)
+        for l in range(w.n_layers):
+            k = synth.on_grid(rng.standard_normal((1, n, w.kv_width), dtype=np.float32), w.storage)
+            v = synth.on_grid(rng.standard_normal((1, n, w.kv_width), dtype=np.float32), w.storage)
+            o.encode_append(l, [0], n, k, v)
+        o.advance([0], n)
+        t += n
+    # sample: `sample_layers` layers of one sequence per step, scaled by batch * n_layers / sample_layers
+    probe_layers = list(range(w.n_layers))
+    times = []
+    sample_layers = None
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        done = 0
+        for l in probe_layers:
+            k = synth.on_grid(rng.standard_normal((1, 1, w.kv_width), dtype=np.float32), w.storage)
+            v = synth.on_grid(rng.standard_normal((1, 1, w.kv_width), dtype=np.float32), w.storage)
+            q = synth.on_grid(rng.standard_normal((1, w.n_q_heads, w.head_dim), dtype=np.float32), w.storage)
+            o.encode_append(l, [0], 1, k, v)
+            o.decode_attention(l, [0], q)
+            done += 1
+            if sample_layers is None and time.perf_counter() - t0 > 120.0 / (args.warmup + args.steps):
+                break
+        if sample_layers is None:
+            sample_layers = done
+            probe_layers = probe_layers[:done]
+        dt = time.perf_counter() - t0
+        if done == w.n_layers:
+            o.advance([0], 1)
+        if i >= args.warmup:
+            times.append(dt * w.batch * w.n_layers / done)
+    ms = 1e3 * float(np.mean(times))
+    value = w.batch / (ms / 1e3)
+    cores = host_threads()
+    sample = (f"per step: encode-append + decode attention of {sample_layers} of {w.n_layers} layers for 1 of "
+              f"{w.batch} sequences at {w.cached_tokens} cached tokens, scaled by the pair count")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.batch, "cached_tokens": w.cached_tokens,
+                       "layers": w.n_layers, "storage": w.storage},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    from paper_2512_06727_b200 import binding as B
+
+    w = workload_of(args)
+    K_, W_ = args.steps, max(args.warmup, 3)
+    n_e2e = 0 if args.no_e2e else max(2, min(K_, 8))
+    extra = 2 * (W_ + K_) + 2 * n_e2e + 4
+    sess, src, aes = build_session(w, args, torch, extra)
+    torch.cuda.set_device(local)
+    sess.device = torch.device(f"cuda:{local}")
+    seqs = list(range(w.batch))
+    do_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
+    keep = tuple(range(min(2, w.batch))) if do_cpu else ()
+    kept = prefill(sess, w, torch, keep)
+    stream = sess.stream()
+    flags = B.INCLUDE_CURRENT_EXACT
+    total_steps = 2 * (W_ + K_)
+    k, v, q, out = step_inputs(sess, w, torch, total_steps)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=sess.device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- pass 1: the headline timing --------------------------------------
+    for i in range(W_):
+        run_step(sess, w, seqs, k, v, q, out, i, stream, flags)
+    sess.ctx.sync_status(stream)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = sess.ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_)]
+    barrier()
+    wall0 = time.perf_counter()
+    for j in range(K_):
+        flush.fill_(j & 0xFF)                      # evict the cache from L2 between steps (outside the event pair)
+        ev[j][0].record()
+        run_step(sess, w, seqs, k, v, q, out, W_ + j, stream, flags)
+        ev[j][1].record()
+    barrier()
+    wall = time.perf_counter() - wall0
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(step_ms))
+    launches = sess.ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    sess.ctx.sync_status(stream)
+    if world > 1:
+        t = torch.tensor([total_ms], device=sess.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K_
+    value = world * w.batch * K_ / (total_ms / 1e3)
+
+    # ---- pass 2: the decode kernel alone, per launch ----------------------
+    base = W_ + K_
+    for i in range(W_):
+        run_step(sess, w, seqs, k, v, q, out, base + i, stream, flags)
+    kev = []
+    cached_at = []
+    for j in range(K_):
+        i = base + W_ + j
+        L = sess.ctx.seq_len(0)
+        for l in range(w.n_layers):
+            sess.ctx.encode_append(l, seqs, 1, k[i, l].data_ptr(), v[i, l].data_ptr(), stream)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            sess.ctx.decode_attention(l, seqs, q[i, l].data_ptr(), out[i, l].data_ptr(), flags, stream)
+            b.record()
+            kev.append((l, L, a, b))
+        sess.ctx.advance(seqs, 1, stream)
+    torch.cuda.synchronize()
+    sess.ctx.sync_status(stream)
+    peaks = measured_peaks()
+    flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
+    byts = sum(sess.ctx.layer_work_per_token(l)[0] * L * w.batch for (l, L, _, _) in kev)
+    kern_ms = sum(a.elapsed_time(b) for (_, _, a, b) in kev)
+    n_k = len(kev)
+    if args.uncompressed:
+        ach = byts / (kern_ms / 1e3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": None}
+    else:
+        ach = flops / (kern_ms / 1e3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None}
+    roof.update({"kernel": "decode_attention (decoder + attention + combine)", "launches": n_k,
+                 "avg_launch_us": 1e3 * kern_ms / n_k, "peak_source": peaks["source"] + " (sustained)",
+                 "algorithmic_flops_per_launch": flops / n_k, "algorithmic_bytes_per_launch": byts / n_k,
+                 "hbm_side_frac": (byts / (kern_ms / 1e3) / 1e9) / peaks["hbm_gbs"]})
+
+    # ---- e2e: host buffers through the C ABI, copies inside the timed region ----
+    e2e = None
+    if n_e2e:
+        hk = [k[0, l].cpu().pin_memory() for l in range(w.n_layers)]
+        hv = [v[0, l].cpu().pin_memory() for l in range(w.n_layers)]
+        hq = [q[0, l].cpu().pin_memory() for l in range(w.n_layers)]
+        ho = [torch.empty_like(hq[l]).pin_memory() for l in range(w.n_layers)]
+
+        def e2e_step():
+            for l in range(w.n_layers):
+                sess.ctx.step_layer_host(l, seqs, hk[l].data_ptr(), hv[l].data_ptr(), hq[l].data_ptr(),
+                                         ho[l].data_ptr(), flags, stream)
+            sess.ctx.advance(seqs, 1, stream)
+            torch.cuda.current_stream().synchronize()      # the step's result is on the host
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_step()
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], device=sess.device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        elem = 2 if w.storage == "bf16" else 4
+        e2e = {"value": world * w.batch * n_e2e / e2e_s, "unit": UNIT, "steps": n_e2e,
+               "h2d_bytes_per_step": w.n_layers * w.batch * (2 * w.kv_width + w.n_q_heads * w.head_dim) * elem,
+               "d2h_bytes_per_step": w.n_layers * w.batch * w.n_q_heads * w.head_dim * elem,
+               "timing": "wall clock around K host-buffer steps, stream synchronised every step"}
+        sess.ctx.sync_status(stream)
+
+    # ---- CPU baseline: the oracle on a bounded sample ------------------------
+    cpu = None
+    if do_cpu and kept:
+        # a fresh decode step at the prefilled length for the sampled sequences, compared with the GPU
+        sess2, _, _ = build_session(w, args, torch, 4)
+        kept2 = prefill(sess2, w, torch, keep)
+        i = 0
+        run_step(sess2, w, seqs, k, v, q, out, i, sess2.stream(), flags)
+        torch.cuda.synchronize()
+        sk = [k[i, l].float().cpu().numpy() for l in range(w.n_layers)]
+        sv = [v[i, l].float().cpu().numpy() for l in range(w.n_layers)]
+        sq = [q[i, l].float().cpu().numpy() for l in range(w.n_layers)]
+        go = [out[i, l].float().cpu().numpy().astype(np.float64) for l in range(w.n_layers)]
+        del sess2
+        r = oracle_sample(w, src, aes, kept2, sk, sv, sq, args.cpu_seconds, go)
+        cpu = {"value": r["value"], "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+               "sample": f"decode step at {w.cached_tokens} cached tokens for {r['pairs']} (sequence, layer) pairs "
+                         f"of {w.batch * w.n_layers} ({r['seconds']:.1f} s), scaled by the pair count",
+               "max_abs_err_gpu_vs_oracle_on_sample": r["max_abs_err_vs_gpu"]}
+
+    if rank == 0:
+        comp, full = sess.ctx.cache_bytes_per_token()
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_, "warmup": W_,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if w.storage == "bf16" else "f32", "data": "synthetic",
+                "config": {"workload": w.name, "batch_per_gpu": w.batch, "cached_tokens": w.cached_tokens,
+                           "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+                           "latent_full": 0 if args.uncompressed else w.latent_full, "reuse_frac": w.reuse_frac,
+                           "page_tokens": w.page_tokens, "kernel": args.kernel,
+                           "uncompressed": bool(args.uncompressed),
+                           "l2": "flushed between steps (256 MiB write outside the per-step event pairs)",
+                           "cache_bytes_per_token": comp, "uncompressed_bytes_per_token": full,
+                           "wall_s_timed_region": wall},
+                "clocks": clocks, "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches)}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
