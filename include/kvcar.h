@@ -200,6 +200,43 @@ kvcar_status kvcar_step_layer_host(kvcar_ctx *ctx, int32_t layer, const int32_t 
                                    const void *k_host, const void *v_host, const void *q_host, void *out_host,
                                    uint32_t flags, void *stream);
 
+/*
+ * kvcar_decode_attention for callers that cannot obtain device memory for the
+ * split-KV scratch.  (The paper has no counterpart to this call; it exists for
+ * integration reasons only.)
+ *
+ * Who needs it: an inference server that gave its whole device budget to its
+ * own arena at start-up and forbids driver allocations afterwards; a plugin
+ * running under a host application that hands it input/output tensors but no
+ * allocator; a latency-critical decode loop in which a cudaMalloc would stall
+ * the device and may fail once memory is fragmented.  Such callers cannot grow
+ * a workspace when a longer sequence needs more partial results.
+ *
+ * What it does: identical arithmetic and kernels to kvcar_decode_attention
+ * (generic kernel family), except that the per-chunk partial results
+ * (max, sum, weighted values) live in a fixed array inside the library image,
+ * KVCAR_STATIC_SCRATCH_BYTES long, which every GPU that loads the library holds
+ * until the process exits.  The call allocates and frees nothing, on the host
+ * side of CUDA or through any library.  q and out are DEVICE buffers as in
+ * kvcar_decode_attention.
+ *
+ * Limits and rules:
+ *  - n_seqs * ceil(longest listed sequence / 128) * n_q_heads * (head_dim + 2)
+ *    floats must fit in KVCAR_STATIC_SCRATCH_BYTES, else KVCAR_ERR_WORKSPACE
+ *    and nothing is launched.
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current, the one whose stream is passed); make that first call
+ *    outside any stream capture.
+ *  - All contexts and streams of a process share the one array per device, and
+ *    it keeps whatever the previous call left; every slot a call reads is
+ *    written earlier in the same call, so nothing needs clearing, but two
+ *    calls that overlap in time on one GPU race on it: keep such calls on one
+ *    stream or order them yourself.
+ */
+#define KVCAR_STATIC_SCRATCH_BYTES (8u << 20)
+kvcar_status kvcar_decode_attention_static(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                           const void *q, void *out, uint32_t flags, void *stream);
+
 /* ---- observability ---------------------------------------------------------- */
 
 /* Reuse table resolution of (layer, kv_head): the layer and head whose cache

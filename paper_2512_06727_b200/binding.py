@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "STATE", 3: "OOM_PAGES", 4: "WORKS
 EXPORTS = [
     "kvcar_create", "kvcar_destroy", "kvcar_set_reuse_map", "kvcar_set_autoencoder", "kvcar_required_bytes",
     "kvcar_bind_memory", "kvcar_set_kernel", "kvcar_seq_open", "kvcar_seq_close", "kvcar_reserve",
-    "kvcar_encode_append", "kvcar_advance", "kvcar_decode_attention", "kvcar_step_layer_host",
+    "kvcar_encode_append", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
+    "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_sync_status",
     "kvcar_last_error",
@@ -81,6 +82,7 @@ def load() -> C.CDLL:
         "kvcar_encode_append": [vp, i32, ip, i32, i32, vp, vp, vp],
         "kvcar_advance": [vp, ip, i32, i32, vp],
         "kvcar_decode_attention": [vp, i32, ip, i32, vp, vp, u32, vp],
+        "kvcar_decode_attention_static": [vp, i32, ip, i32, vp, vp, u32, vp],
         "kvcar_step_layer_host": [vp, i32, ip, i32, vp, vp, vp, vp, u32, vp],
         "kvcar_debug_resolve": [vp, i32, i32, i32, ip, ip, ip],
         "kvcar_debug_locate": [vp, i32, i32, ip, C.POINTER(C.c_int64)],
@@ -205,6 +207,13 @@ class Context:
     def decode_attention(self, layer: int, seqs: Sequence[int], q: int, out: int,
                          flags: int = INCLUDE_CURRENT_EXACT, stream: int = 0):
         self._check(self.lib.kvcar_decode_attention(self._h, layer, self._seqs(seqs), len(seqs), q, out, flags, stream))
+
+    def decode_attention_static(self, layer: int, seqs: Sequence[int], q: int, out: int,
+                                flags: int = INCLUDE_CURRENT_EXACT, stream: int = 0):
+        """Decode attention whose split-KV scratch is the library's built-in array
+        (allocates nothing; see kvcar_decode_attention_static in kvcar.h)."""
+        self._check(self.lib.kvcar_decode_attention_static(self._h, layer, self._seqs(seqs), len(seqs), q, out,
+                                                           flags, stream))
 
     def step_layer_host(self, layer: int, seqs: Sequence[int], k_host: int, v_host: int, q_host: int,
                         out_host: int, flags: int = INCLUDE_CURRENT_EXACT, stream: int = 0):

@@ -775,3 +775,95 @@ kvcar_status kvcar_sync_status(kvcar_ctx *c, void *stream) {
 const char *kvcar_last_error(kvcar_ctx *c) { return c ? c->err.c_str() : "null context"; }
 
 }  // extern "C"
+
+// =============================================================================
+// Allocation-free decode attention: split-KV partials in a fixed array that is
+// part of the library image.  In host code `g_static_scratch` is only a handle
+// for the runtime, never an address a kernel may use: the device address is
+// looked up once per device with cudaGetSymbolAddress and that pointer is what
+// the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[KVCAR_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float *g_static_scratch_ptr[kMaxDevices] = {};  // per device; filled on the first call there
+
+// Device address of the scratch array on the current device (set-up on first use).
+cudaError_t static_scratch_for_current_device(float **out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    float *p = __atomic_load_n(&g_static_scratch_ptr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        void *sym = nullptr;
+        e = cudaGetSymbolAddress(&sym, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        p = reinterpret_cast<float *>(sym);
+        __atomic_store_n(&g_static_scratch_ptr[dev], p, __ATOMIC_RELEASE);  // same value from any thread
+    }
+    *out = p;
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" kvcar_status kvcar_decode_attention_static(kvcar_ctx *c, int32_t layer, const int32_t *seqs,
+                                                      int32_t n_seqs, const void *q, void *out, uint32_t flags,
+                                                      void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (layer < 0 || layer >= c->cfg.n_layers || !q || !out)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
+    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    if (flags & ~KVCAR_INCLUDE_CURRENT_EXACT) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    const kvcar_config &g = c->cfg;
+    int max_len = 0;
+    for (int i = 0; i < n_seqs; ++i) max_len = std::max(max_len, c->len[seqs[i]]);
+    const int chunk_tokens = 128;
+    const int n_chunks = (max_len + chunk_tokens - 1) / chunk_tokens;
+    const size_t need = (size_t)n_seqs * std::max(n_chunks, 1) * g.n_q_heads * (g.head_dim + 2) * sizeof(float);
+    if (need > (size_t)KVCAR_STATIC_SCRATCH_BYTES) {
+        char buf[160];
+        snprintf(buf, sizeof buf, "static scratch too small: this call needs %zu bytes of split-KV partials, the "
+                 "built-in array holds %u", need, (unsigned)KVCAR_STATIC_SCRATCH_BYTES);
+        return fail(c, KVCAR_ERR_WORKSPACE, buf);
+    }
+    if (decode_generic_smem(g.n_q_heads, g.head_dim, c->max_d, c->max_m) > 227 * 1024)
+        return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");
+    float *scratch = nullptr;
+    cudaError_t e = static_scratch_for_current_device(&scratch);
+    if (e != cudaSuccess) return cuda_fail(c, e, "address of the built-in scratch array");
+    cudaStream_t st = (cudaStream_t)stream;
+    kvcar_status s = flush_tables(c, st);
+    if (s != KVCAR_OK) return s;
+    DecodeArgs a{};
+    a.plan = reinterpret_cast<const LayerPlan *>(c->weights + c->plan_off) + layer;
+    a.block_table = reinterpret_cast<const int32_t *>(c->ws + c->bt_off);
+    a.seq_len = reinterpret_cast<const int32_t *>(c->ws + c->len_off);
+    a.q = q;
+    a.out = out;
+    a.partials = scratch;
+    a.status = reinterpret_cast<int32_t *>(c->ws + c->status_off);
+    a.max_pages_per_seq = g.max_pages_per_seq;
+    a.page_tokens = g.page_tokens;
+    a.hq = g.n_q_heads;
+    a.hkv = g.n_kv_heads;
+    a.hd = g.head_dim;
+    a.chunk_tokens = chunk_tokens;
+    a.max_chunks = std::max(n_chunks, 1);  // partials are packed for this call's longest sequence
+    a.flags = flags;
+    a.scale = 1.0f / std::sqrt((float)g.head_dim);
+    SeqList sl;
+    sl.n = n_seqs;
+    memcpy(sl.id, seqs, (size_t)n_seqs * 4);
+    if (n_chunks > 0) {
+        e = launch_decode_generic(a, sl, g.storage, c->max_d, c->max_m, n_chunks, st);
+        if (e != cudaSuccess) return cuda_fail(c, e, "decode launch");
+        ++c->launches;
+    }
+    e = launch_combine(a, sl, g.storage, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "combine launch");
+    ++c->launches;
+    return KVCAR_OK;
+}
