@@ -261,6 +261,9 @@ kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *ctx, double *compressed, dou
 kvcar_status kvcar_layer_work_per_token(kvcar_ctx *ctx, int32_t layer, double *bytes, double *flops);
 /* Number of kernels the library has launched so far on this context. */
 kvcar_status kvcar_launch_count(kvcar_ctx *ctx, int64_t *count);
+/* Kernel family (kvcar_kernel: GENERIC or TENSOR) that kvcar_decode_attention will use
+ * for `layer` under the current kvcar_set_kernel choice.  Only after kvcar_bind_memory. */
+kvcar_status kvcar_layer_kernel(kvcar_ctx *ctx, int32_t layer, int32_t *kernel);
 /* Synchronise `stream` and report any asynchronous CUDA error or device-side
  * bounded-wait timeout recorded since the last call. */
 kvcar_status kvcar_sync_status(kvcar_ctx *ctx, void *stream);

@@ -29,7 +29,7 @@ EXPORTS = [
     "kvcar_encode_append", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
     "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
-    "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_sync_status",
+    "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
     "kvcar_last_error",
 ]
 
@@ -91,6 +91,7 @@ def load() -> C.CDLL:
         "kvcar_cache_bytes_per_token": [vp, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "kvcar_layer_work_per_token": [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "kvcar_launch_count": [vp, C.POINTER(C.c_int64)],
+        "kvcar_layer_kernel": [vp, i32, ip],
         "kvcar_sync_status": [vp, vp],
     }
     for name, args in sig.items():
@@ -255,6 +256,11 @@ class Context:
         n = C.c_int64()
         self._check(self.lib.kvcar_launch_count(self._h, C.byref(n)))
         return n.value
+
+    def layer_kernel(self, layer: int) -> int:
+        k = C.c_int32()
+        self._check(self.lib.kvcar_layer_kernel(self._h, layer, C.byref(k)))
+        return k.value
 
     def sync_status(self, stream: int = 0):
         self._check(self.lib.kvcar_sync_status(self._h, stream))

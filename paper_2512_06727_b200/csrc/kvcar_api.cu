@@ -51,7 +51,7 @@ struct kvcar_ctx {
     std::vector<size_t> pool_off, cur_off;  // [layer*2+which]
     std::vector<int> width;                 // elements per row
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
-    size_t plan_off = 0, enc_off = 0;       // inside weights
+    size_t plan_off = 0, enc_off = 0, tmap_off = 0;  // inside weights
     size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0;  // inside workspace
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
@@ -141,6 +141,8 @@ void compute_layout(kvcar_ctx *c) {
     w = align_up(w + (size_t)nl * sizeof(LayerPlan), 256);
     c->enc_off = w;
     w = align_up(w + (size_t)nl * 2 * sizeof(EncPlan), 256);
+    c->tmap_off = w;  // TMA descriptors of the tensor-core kernel: pool, decoder FC1, decoder FC2 per (layer, which)
+    w = align_up(w + (size_t)nl * 2 * 3 * 128, 256);
     c->weights_bytes = w;
 
     // workspace
@@ -464,6 +466,9 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
             }
         }
     }
+    // tensor maps and per-source pointers to them (fills the tmap region of the image, edits `plans`)
+    tc_setup(c->tc, c->cfg, plans, nl, c->weights, c->tmap_off, img.data(), (size_t)g.max_pages * g.page_tokens,
+             c->width.data());
     memcpy(&img[c->plan_off], plans, (size_t)nl * sizeof(LayerPlan));
 
     std::vector<EncPlan> enc(nl * 2);
@@ -505,7 +510,6 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
         for (size_t i = 0; i < c->table[s].size(); ++i) c->pending.push_back(make_int4(0, s, (int)i, c->table[s][i]));
         if (c->len[s]) c->pending.push_back(make_int4(1, s, 0, c->len[s]));
     }
-    tc_setup(c->tc, c->cfg, plans, nl, (const LayerPlan *)(c->weights + c->plan_off), (size_t)g.max_pages * g.page_tokens);
     return KVCAR_OK;
 }
 
@@ -751,6 +755,13 @@ kvcar_status kvcar_layer_work_per_token(kvcar_ctx *c, int32_t layer, double *byt
 kvcar_status kvcar_launch_count(kvcar_ctx *c, int64_t *count) {
     if (!c || !count) return KVCAR_ERR_INVALID_ARG;
     *count = c->launches;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_layer_kernel(kvcar_ctx *c, int32_t layer, int32_t *kernel) {
+    if (!c || !kernel || layer < 0 || layer >= c->cfg.n_layers) return fail(c, KVCAR_ERR_INVALID_ARG, "bad argument");
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    *kernel = (use_tensor_kernel(c) && tc_layer_supported(c->tc, layer)) ? KVCAR_KERNEL_TENSOR : KVCAR_KERNEL_GENERIC;
     return KVCAR_OK;
 }
 

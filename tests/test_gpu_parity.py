@@ -52,6 +52,8 @@ def test_gpt2_shape_stack_bf16_with_reuse(kernel):
     p.prefill([0], 131)
     p.prefill([3], 64)
     p.check_latents(seqs)
+    if kernel == B.KERNEL_AUTO:     # the bf16 stack must really run on the tensor-core kernel
+        assert all(p.s.ctx.layer_kernel(l) == B.KERNEL_TENSOR for l in range(w.n_layers))
     for step in range(2):
         _check_step(p.decode_step(seqs, step), "bf16", f"step {step}")
     p.check_latents(seqs)
@@ -71,6 +73,8 @@ def test_tinyllama_shape_gqa_stack_bf16_with_reuse(kernel):
     for s, n in zip(seqs, (300, 257, 128, 1)):
         p.prefill([s], n)
     p.check_latents(seqs)
+    if kernel == B.KERNEL_AUTO:
+        assert all(p.s.ctx.layer_kernel(l) == B.KERNEL_TENSOR for l in range(w.n_layers))
     for step in range(2):
         _check_step(p.decode_step(seqs, step), "bf16", f"step {step}")
 
