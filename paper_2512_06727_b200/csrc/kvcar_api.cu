@@ -136,6 +136,7 @@ void compute_layout(kvcar_ctx *c) {
         w = align_up(w + 2 * mats * c->elem, 256);                                 // transposed enc + dec
         w = align_up(w + (size_t)(4 * a.hidden + a.latent + a.in_dim) * sizeof(float), 256);  // s,t x2, b2 x2
         if (g.storage == KVCAR_BF16) w = align_up(w + mats * 2, 256);             // K-major decoder copies
+        w = align_up(w + mats * c->elem, 256);                                     // row-major encoder copies
     }
     c->plan_off = w;
     w = align_up(w + (size_t)nl * sizeof(LayerPlan), 256);
@@ -377,7 +378,7 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
 
     std::vector<char> img(c->weights_bytes, 0);
     struct Packed {
-        size_t enc_w1t, enc_w2t, dec_w1t, dec_w2t, enc_s, enc_t, enc_b2, dec_s, dec_t, dec_b2, w1k, w2k;
+        size_t enc_w1t, enc_w2t, dec_w1t, dec_w2t, enc_s, enc_t, enc_b2, dec_s, dec_t, dec_b2, w1k, w2k, enc_w1r, enc_w2r;
     };
     std::vector<Packed> pk(nl * 2);
     size_t w = 0;
@@ -413,6 +414,11 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
             put_elems(&img[p.w1k], a.dec_w1.data(), M * D, KVCAR_BF16);
             put_elems(&img[p.w2k], a.dec_w2.data(), I * M, KVCAR_BF16);
         }
+        p.enc_w1r = w;
+        p.enc_w2r = p.enc_w1r + M * I * E;
+        w = align_up(w + (M * I + D * M) * E, 256);
+        put_elems(&img[p.enc_w1r], a.enc_w1.data(), M * I, g.storage);
+        put_elems(&img[p.enc_w2r], a.enc_w2.data(), D * M, g.storage);
     }
 
     // per-layer decode plans
@@ -490,6 +496,8 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
             e.slope = a.slope;
             e.w1t = c->weights + pk[i].enc_w1t;
             e.w2t = c->weights + pk[i].enc_w2t;
+            e.w1r = c->weights + pk[i].enc_w1r;
+            e.w2r = c->weights + pk[i].enc_w2r;
             e.s1 = (const float *)(c->weights + pk[i].enc_s);
             e.t1 = (const float *)(c->weights + pk[i].enc_t);
             e.b2 = (const float *)(c->weights + pk[i].enc_b2);
@@ -574,7 +582,16 @@ kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seq
     SeqList sl;
     sl.n = n_seqs;
     memcpy(sl.id, seqs, (size_t)n_seqs * 4);
-    cudaError_t e = launch_encode_generic(a, sl, c->cfg.storage, c->max_in, c->max_m, st);
+    // one token per sequence: the cluster kernel that splits the weight stream over 8 SMs per 8 rows
+    // (needs 16-byte loadable weight rows and fits its two row blocks in default shared memory)
+    const int vl = 16 / c->elem;
+    bool cluster_ok = n_tokens == 1 && (size_t)8 * (c->max_in + c->max_m) * sizeof(float) <= 200 * 1024;
+    for (int w = 0; w < 2 && cluster_ok; ++w) {
+        const AEHost &ae = c->ae[layer * 2 + w];
+        if (ae.set && (ae.in_dim % vl || ae.hidden % vl)) cluster_ok = false;
+    }
+    cudaError_t e = cluster_ok ? launch_encode_cluster(a, sl, c->cfg.storage, c->max_in, c->max_m, st)
+                               : launch_encode_generic(a, sl, c->cfg.storage, c->max_in, c->max_m, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "encode launch");
     ++c->launches;
     return KVCAR_OK;

@@ -56,6 +56,8 @@ struct EncPlan {
     const float *s1, *t1;
     const void *w2t;  // encoder FC2 transposed [m][d]
     const float *b2;
+    const void *w1r;  // encoder FC1 as given, [m][in_dim], storage dtype (rows read by one warp each)
+    const void *w2r;  // encoder FC2 as given, [d][m]
     int32_t width, d, m, in_dim, compressed, n_stored;
     float slope;
     int32_t pad_;
@@ -101,6 +103,9 @@ struct TableUpdates {
 // launchers implemented in kvcar_generic.cu (return cudaGetLastError())
 cudaError_t launch_table_updates(int32_t *block_table, int32_t *seq_len, const TableUpdates &u, cudaStream_t st);
 cudaError_t launch_encode_generic(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m,
+                                  cudaStream_t st);
+// cluster kernel for one new token per sequence (kvcar_encode.cu)
+cudaError_t launch_encode_cluster(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m,
                                   cudaStream_t st);
 cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int dtype, int max_d, int max_m,
                                   int grid_chunks, cudaStream_t st);
