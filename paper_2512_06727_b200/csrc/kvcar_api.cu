@@ -51,7 +51,7 @@ struct kvcar_ctx {
     std::vector<size_t> pool_off, cur_off;  // [layer*2+which]
     std::vector<int> width;                 // elements per row
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
-    size_t plan_off = 0, enc_off = 0, tmap_off = 0;  // inside weights
+    size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
     size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0;  // inside workspace
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
@@ -144,6 +144,8 @@ void compute_layout(kvcar_ctx *c) {
     w = align_up(w + (size_t)nl * 2 * sizeof(EncPlan), 256);
     c->tmap_off = w;  // TMA descriptors of the tensor-core kernel: pool, decoder FC1, decoder FC2 per (layer, which)
     w = align_up(w + (size_t)nl * 2 * 3 * 128, 256);
+    c->tcpart_off = w;  // per-layer job tables of the tensor-core kernel
+    w = align_up(w + tc_part_bytes(nl), 256);
     c->weights_bytes = w;
 
     // workspace
@@ -472,9 +474,9 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
             }
         }
     }
-    // tensor maps and per-source pointers to them (fills the tmap region of the image, edits `plans`)
-    tc_setup(c->tc, c->cfg, plans, nl, c->weights, c->tmap_off, img.data(), (size_t)g.max_pages * g.page_tokens,
-             c->width.data());
+    // tensor maps and job tables of the tensor-core kernel (fills their regions of the image)
+    tc_setup(c->tc, c->cfg, plans, nl, c->weights, c->tmap_off, c->tcpart_off, img.data(),
+             (size_t)g.max_pages * g.page_tokens);
     memcpy(&img[c->plan_off], plans, (size_t)nl * sizeof(LayerPlan));
 
     std::vector<EncPlan> enc(nl * 2);
@@ -654,7 +656,9 @@ kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *
             return fail(c, KVCAR_ERR_UNSUPPORTED, std::string("tensor-core kernel cannot run this layer: ") + c->tc.why);
         cudaError_t e;
         if (want_tc) {
-            e = tc_launch_decode(c->tc, a, sl, layer, n_chunks, st);
+            int32_t lens[KVCAR_MAX_BATCH];
+            for (int i = 0; i < n_seqs; ++i) lens[i] = c->len[seqs[i]];
+            e = tc_launch_decode(c->tc, a, sl, lens, layer, st);
         } else {
             if (decode_generic_smem(a.hq, a.hd, c->max_d, c->max_m) > 227 * 1024)
                 return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");

@@ -23,9 +23,6 @@ struct SourcePlan {
     const float *b2;   // [in_dim]
     const void *w1k;   // K-major bf16 copies for the tensor-core kernel: [m][d]
     const void *w2k;   //                                                  [in_dim][m]
-    const void *tm_pool;  // TMA descriptors (device memory, 128 B each) of pool, w1k, w2k; null if unavailable
-    const void *tm_w1;
-    const void *tm_w2;
     int32_t width;     // elements per pool row (= d if compressed, = in_dim if raw)
     int32_t d, m, in_dim;
     int32_t compressed;

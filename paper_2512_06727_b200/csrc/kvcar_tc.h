@@ -5,30 +5,70 @@
 namespace kvcar {
 
 constexpr int TC_MAX_LAYERS = 512;
+constexpr int TC_MAX_SRC = 6;    // distinct source layers per K or V of one head subset
+constexpr int TC_MAX_JOBS = 24;  // accumulator jobs per K or V of one head subset
+constexpr int TC_MAX_SPLIT = 4;  // a layer's KV heads can be split over up to 4 clusters per tile pair
+
+// One source layer as the tensor-core kernel sees it.
+struct TcSrc {
+    const void *tm_pool, *tm_w1, *tm_w2;  // TMA descriptors (device memory): cache rows, decoder FC1, decoder FC2
+    const float *s1, *t1, *b2;            // fused bias+BatchNorm scale/shift [m]; last-FC bias [in_dim]
+    int32_t d, m;
+    float slope;
+    int32_t in_dim;
+};
+
+// One accumulator job: a chunk of hidden columns (first decoder layer) or a group of
+// up to four restored heads (second decoder layer).  The TMA producer, the MMA issuer
+// and the epilogue warps all walk the same list in the same order.
+struct TcJob {
+    uint8_t kind;    // 1 = hidden chunk, 2 = head group
+    uint8_t src;     // index into TcPart::src[which]
+    uint8_t nh;      // head group: real heads (1..4)
+    uint8_t first;   // first job of its source
+    uint16_t c0;     // hidden chunk: first hidden column
+    uint16_t nc;     // hidden chunk: width (multiple of 16, <= 256)
+    int8_t kvh[4];   // head group: KV head of the reading layer per head place (-1 = padding)
+    int8_t slot[4];  // head group: 64-wide column slot of the restored row per head place
+};
+
+// Everything one cluster needs for one layer and one subset of its KV heads.
+struct TcPart {
+    int32_t n_src[2], n_jobs[2];
+    int32_t h_lo, h_hi;  // KV heads [h_lo, h_hi) of the reading layer
+    int32_t max_m, pad_;
+    TcSrc src[2][TC_MAX_SRC];
+    TcJob jobs[2][TC_MAX_JOBS];
+};
 
 struct TcLayerCfg {
-    uint8_t ok;        // this layer can run on the tensor-core kernel
-    uint8_t nslot;     // operand ring depth (16 KB slots)
-    uint16_t max_m;    // widest hidden layer among the layer's sources
-    uint16_t max_in;   // most restored columns (needed heads x 64) of one source
-    uint32_t smem;     // dynamic shared memory per CTA
+    uint8_t ok;            // this layer can run on the tensor-core kernel
+    uint8_t split_ok[3];   // head splits 1, 2, 4 available
+    uint16_t max_m;        // widest hidden layer among the layer's sources
+    uint16_t max_in;       // widest restored row among the layer's sources
 };
 
 struct TcState {
     bool available = false;
     const char *why = "not set up";
+    char *parts_dev = nullptr;  // TcPart[n_layers][7] in the weights buffer: split 1 -> [0], 2 -> [1..2], 4 -> [3..6]
+    int n_sms = 148;
     TcLayerCfg layer[TC_MAX_LAYERS];
 };
 
-// Build the TMA descriptors into the host image of the weights buffer (at tmap_off),
-// point every SourcePlan at its three descriptors and decide per layer whether the
-// tensor-core kernel can run it.  Never fails hard: on any problem the state stays
-// unavailable with a reason and the generic kernels run.
-void tc_setup(TcState &tc, const kvcar_config &cfg, LayerPlan *plans_host, int n_layers, char *weights_dev,
-              size_t tmap_off, char *weights_img, size_t pool_rows, const int *pool_width);
+// bytes of the per-layer job tables inside the weights buffer
+size_t tc_part_bytes(int n_layers);
+
+// Build the TMA descriptors and the per-layer job tables into the host image of the
+// weights buffer (at tmap_off / part_off) and decide per layer whether the tensor-core
+// kernel can run it.  Never fails hard: on any problem the state stays unavailable
+// with a reason and the generic kernels run.
+void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans_host, int n_layers, char *weights_dev,
+              size_t tmap_off, size_t part_off, char *weights_img, size_t pool_rows);
 void tc_destroy(TcState &tc);
 bool tc_layer_supported(const TcState &tc, int layer);
-cudaError_t tc_launch_decode(const TcState &tc, const DecodeArgs &a, const SeqList &seqs, int layer, int n_chunks,
-                             cudaStream_t st);
+// lens: host copy of the listed sequences' lengths (same values the device table holds)
+cudaError_t tc_launch_decode(const TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
+                             int layer, cudaStream_t st);
 
 }  // namespace kvcar
