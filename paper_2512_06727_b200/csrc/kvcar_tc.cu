@@ -73,6 +73,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
+// same, ordering only this CTA's earlier operations (enough where the data handed over is tensor memory already
+// read, or this CTA's shared memory already fenced for the async proxy)
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -124,6 +129,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int 
         "[%4];" ::"r"(dst),
         "l"(tmap), "r"(x), "r"(y), "r"(cluster_bar)
         : "memory");
+}
+
+// bring one box of a tensor into L2 ahead of its load
+__device__ __forceinline__ void tma_prefetch_2d(const void *tmap, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -303,18 +313,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 
     if (warp == 0) {
         // ============================== TMA producer (both CTAs) ==============================
-        if (lane == 0) {
-            // pool rows of the tile's two 64-token halves (a half with no valid token re-reads a valid row block)
-            int row[2] = {0, 0};
-            if (mine.valid > 0) {
-                const int seq = seqs.id[mine.si];
-                for (int h = 0; h < 2; ++h) {
-                    int t = mine.chunk * TILE + 64 * h;
-                    if (64 * h >= mine.valid) t = mine.chunk * TILE;
-                    const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
-                    row[h] = page * a.page_tokens + t % a.page_tokens;
-                }
+        // pool rows of the tile's two 64-token halves (a half with no valid token re-reads a valid row block)
+        int row[2] = {0, 0};
+        if (mine.valid > 0) {
+            const int seq = seqs.id[mine.si];
+            for (int h = 0; h < 2; ++h) {
+                int t = mine.chunk * TILE + 64 * h;
+                if (64 * h >= mine.valid) t = mine.chunk * TILE;
+                const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
+                row[h] = page * a.page_tokens + t % a.page_tokens;
             }
+        }
+        if (lane > 0 && mine.valid > 0) {
+            // the other lanes pull this tile's latent rows of every source from HBM into L2 ahead of the loads
+            int item = 0;
+            for (int which = 0; which < 2; ++which)
+                for (int sidx = 0; sidx < P.n_src[which]; ++sidx) {
+                    const TcSrc &sp = P.src[which][sidx];
+                    const int n = 2 * ((sp.d + 63) >> 6);
+                    for (int i = 0; i < n; ++i, ++item)
+                        if (item % 31 == lane - 1 && (i & 1) * 64 < mine.valid)
+                            tma_prefetch_2d(sp.tm_pool, (i >> 1) * 64, row[i & 1]);
+                }
+        }
+        if (lane == 0) {
             uint32_t slot = 0, phase = 0;
             // wait for the slot to be free in this CTA, announce the pair's bytes (leader), return the slot
             auto acquire = [&](uint32_t pair_bytes) -> uint32_t {
@@ -432,7 +454,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         const uint32_t lane_base = 32u * (warp & 3);  // TMEM lane quarter this warp may read
         const int row = lane_base + lane;             // accumulator row of this thread
         const uint32_t tl_addr = lane_base << 16;
-        float *s1 = fparam, *t1 = fparam + lay.max_m, *b2 = fparam + 2 * lay.max_m;
+        const int m_pad = (lay.max_m + 31) & ~31;  // scale/shift rows are read in whole 32-column groups
+        float *s1 = fparam, *t1 = fparam + m_pad, *b2 = fparam + 2 * m_pad;
         const uint32_t jempty_leader[2] = {map_to_cta(B.jempty, 0), map_to_cta(B.jempty + 8, 0)};
         const uint32_t hid_leader = map_to_cta(B.hid_ready, 0);
         const uint32_t peer_S = map_to_cta(smem_u32(Sall), rank ^ 1u);
@@ -465,15 +488,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (job.kind == 1) {
                     if (job.first) {
                         epi_bar_sync();  // everyone is done with the previous source's parameters
-                        for (int i = et; i < m; i += 256) {
-                            s1[i] = sp.s1[i];
-                            t1[i] = sp.t1[i];
+                        for (int i = et; i < m_pad; i += 256) {
+                            s1[i] = i < m ? sp.s1[i] : 0.f;
+                            t1[i] = i < m ? sp.t1[i] : 0.f;
                         }
                         for (int i = et; i < sp.in_dim; i += 256) b2[i] = sp.b2[i];
                         epi_bar_sync();
                     }
                     // ---- bias + BatchNorm + LeakyReLU, bf16, into the swizzled hidden slabs ----
-                    const float slope = sp.slope;
+                    const float2 slope2 = make_float2(sp.slope, sp.slope);
+                    const bool lr_max = sp.slope <= 1.f;
                     mbar_wait(B.jfull + 8 * buf, (jc >> 1) & 1u, a.status, &abort_flag, 0x301);
                     tc_fence_after();
                     const int ngroups = (job.nc + 31) >> 5;
@@ -482,11 +506,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         tmem_ld32(acc + 32u * g, v);
                         tmem_ld_wait();
                         const int col0 = job.c0 + 32 * g;
+                        const float4 *s4 = reinterpret_cast<const float4 *>(s1 + col0);  // padded to 32 columns
+                        const float4 *t4 = reinterpret_cast<const float4 *>(t1 + col0);
 #pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) {
-                            const int col = min(col0 + jj, m - 1);
-                            const float x = fmaf(v[jj], s1[col], t1[col]);
-                            v[jj] = fmaxf(x, 0.f) + slope * fminf(x, 0.f);
+                        for (int q8 = 0; q8 < 8; ++q8) {
+                            const float4 sv = s4[q8], tv = t4[q8];
+                            const float2 x0 = __ffma2_rn(make_float2(v[4 * q8], v[4 * q8 + 1]), make_float2(sv.x, sv.y),
+                                                         make_float2(tv.x, tv.y));
+                            const float2 x1 = __ffma2_rn(make_float2(v[4 * q8 + 2], v[4 * q8 + 3]),
+                                                         make_float2(sv.z, sv.w), make_float2(tv.z, tv.w));
+                            const float2 y0 = __fmul2_rn(x0, slope2), y1 = __fmul2_rn(x1, slope2);
+                            // LeakyReLU: the larger of x and slope*x for slope <= 1, the smaller for slope > 1
+                            v[4 * q8 + 0] = lr_max ? fmaxf(x0.x, y0.x) : fminf(x0.x, y0.x);
+                            v[4 * q8 + 1] = lr_max ? fmaxf(x0.y, y0.y) : fminf(x0.y, y0.y);
+                            v[4 * q8 + 2] = lr_max ? fmaxf(x1.x, y1.x) : fminf(x1.x, y1.x);
+                            v[4 * q8 + 3] = lr_max ? fmaxf(x1.y, y1.y) : fminf(x1.y, y1.y);
                         }
                         // 32 columns = 4 chunks of 16 B inside slab (col0 / 64)
                         const uint32_t slab = s_hidden + (uint32_t)(col0 >> 6) * SLOT_BYTES + (uint32_t)row * 128u;
@@ -509,8 +543,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        mbar_arrive_cluster(jempty_leader[buf]);
-                        mbar_arrive_cluster(hid_leader + 8u * (uint32_t)(job.c0 >> 8));
+                        mbar_arrive_remote(jempty_leader[buf]);
+                        mbar_arrive_remote(hid_leader + 8u * (uint32_t)(job.c0 >> 8));
                     }
                     continue;
                 }
@@ -525,30 +559,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         tmem_ld32(acc + 64u * hp, y);
                         tmem_ld32(acc + 64u * hp + 32u, y + 32);
                         tmem_ld_wait();
-                        const float *bb = b2 + job.slot[hp] * 64;
+                        const float4 *bb = reinterpret_cast<const float4 *>(b2 + job.slot[hp] * 64);
+                        float2 y2[32];
 #pragma unroll
-                        for (int c = 0; c < 64; c += 4) {
-                            const float4 b4 = *reinterpret_cast<const float4 *>(bb + c);
-                            y[c] += b4.x; y[c + 1] += b4.y; y[c + 2] += b4.z; y[c + 3] += b4.w;
+                        for (int c = 0; c < 16; ++c) {
+                            const float4 b4 = bb[c];
+                            y2[2 * c] = __fadd2_rn(make_float2(y[4 * c], y[4 * c + 1]), make_float2(b4.x, b4.y));
+                            y2[2 * c + 1] = __fadd2_rn(make_float2(y[4 * c + 2], y[4 * c + 3]), make_float2(b4.z, b4.w));
                         }
                         const int ql0 = (job.kvh[hp] - h_lo) * group;
                         for (int g = 0; g < group; ++g) {
                             const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g) * 64);
-                            float dot = 0.f;
+                            float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
 #pragma unroll
                             for (int c = 0; c < 16; ++c) {
                                 const float4 qq = q4[c];
-                                dot = fmaf(y[4 * c + 0], qq.x, dot);
-                                dot = fmaf(y[4 * c + 1], qq.y, dot);
-                                dot = fmaf(y[4 * c + 2], qq.z, dot);
-                                dot = fmaf(y[4 * c + 3], qq.w, dot);
+                                d0 = __ffma2_rn(y2[2 * c], make_float2(qq.x, qq.y), d0);
+                                d1 = __ffma2_rn(y2[2 * c + 1], make_float2(qq.z, qq.w), d1);
                             }
+                            const float dot = (d0.x + d0.y) + (d1.x + d1.y);
                             Smine[(ql0 + g) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
                         }
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(jempty_leader[buf]);
+                    if (lane == 0) mbar_arrive_remote(jempty_leader[buf]);
                     epi_bar_sync();
                     // tile softmax of the job's query heads; probabilities go to both CTAs
                     if (mine.valid > 0) {
@@ -591,30 +626,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     if (kvh >= 0 && tt.valid > 0) {
                         const int ql0 = (kvh - h_lo) * group;
                         const float *Sp = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE;
-                        float accv[8];
+                        float2 accv[8];
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) accv[g] = 0.f;
+                        for (int g = 0; g < 8; ++g) accv[g] = make_float2(0.f, 0.f);
                         for (int gi = 0; gi < 4; ++gi) {
                             if (32 * gi >= tt.valid) break;
                             float y[32];
                             tmem_ld32(acc + 128u * chalf + 32u * gi, y);
                             tmem_ld_wait();
+                            if (32 * gi + 32 > tt.valid) {  // rows past the tile's end may hold anything
 #pragma unroll
-                            for (int t = 0; t < 32; ++t) y[t] = (32 * gi + t < tt.valid) ? y[t] : 0.f;
+                                for (int t = 0; t < 32; ++t) y[t] = (32 * gi + t < tt.valid) ? y[t] : 0.f;
+                            }
 #pragma unroll
                             for (int g = 0; g < 8; ++g) {
                                 if (g < group) {
                                     const float4 *p4 = reinterpret_cast<const float4 *>(Sp + g * PSTRIDE + 32 * gi);
-                                    float s = accv[g];
+                                    float2 s0 = accv[g], s1v = make_float2(0.f, 0.f);
 #pragma unroll
                                     for (int t = 0; t < 8; ++t) {
                                         const float4 pp = p4[t];
-                                        s = fmaf(pp.x, y[4 * t + 0], s);
-                                        s = fmaf(pp.y, y[4 * t + 1], s);
-                                        s = fmaf(pp.z, y[4 * t + 2], s);
-                                        s = fmaf(pp.w, y[4 * t + 3], s);
+                                        s0 = __ffma2_rn(make_float2(pp.x, pp.y), make_float2(y[4 * t], y[4 * t + 1]), s0);
+                                        s1v = __ffma2_rn(make_float2(pp.z, pp.w), make_float2(y[4 * t + 2], y[4 * t + 3]), s1v);
                                     }
-                                    accv[g] = s;
+                                    accv[g] = __fadd2_rn(s0, s1v);
                                 }
                             }
                         }
@@ -624,13 +659,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             if (g < group) {
                                 const int qh = (h_lo * group) + ql0 + g;
                                 float *part = a.partials + (((int64_t)tt.si * a.max_chunks + tt.chunk) * hq + qh) * (64 + 2);
-                                part[2 + c] = accv[g] + bias * Sp[g * PSTRIDE + 128];
+                                part[2 + c] = (accv[g].x + accv[g].y) + bias * Sp[g * PSTRIDE + 128];
                             }
                         }
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(jempty_leader[buf]);
+                    if (lane == 0) mbar_arrive_remote(jempty_leader[buf]);
                 }
             }
         }
@@ -689,7 +724,7 @@ PairLaunch make_launch(int nq_local, int max_m, int max_in, int nslot) {
     l.off_part = o;
     o = up(o + (uint32_t)sizeof(TcPart), 16);
     l.off_fparam = o;
-    o = up(o + (uint32_t)(2 * max_m + max_in) * 4, 16);
+    o = up(o + (uint32_t)(2 * ((max_m + 31) & ~31) + max_in) * 4, 16);
     l.off_q = o;
     o = up(o + (uint32_t)nq_local * 64 * 4, 16);
     l.off_s = o;
