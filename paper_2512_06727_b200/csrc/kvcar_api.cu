@@ -52,7 +52,7 @@ struct kvcar_ctx {
     std::vector<int> width;                 // elements per row
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
     size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
-    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0;  // inside workspace
+    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0;  // inside workspace
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
     std::vector<LayerPlan> plans_host;
@@ -164,6 +164,8 @@ void compute_layout(kvcar_ctx *c) {
     s = align_up(s + (size_t)nb * c->max_chunks * g.n_q_heads * (g.head_dim + 2) * sizeof(float), 256);
     c->stage_off = s;
     s = align_up(s + (size_t)nb * (2 * W + 2 * g.n_q_heads * g.head_dim) * c->elem + 4 * 256, 256);
+    c->enchid_off = s;  // hidden activations between the two decode-time encoder launches
+    s = align_up(s + (size_t)2 * nb * c->max_m * sizeof(float), 256);
     c->ws_bytes = s;
 }
 
@@ -584,18 +586,20 @@ kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seq
     SeqList sl;
     sl.n = n_seqs;
     memcpy(sl.id, seqs, (size_t)n_seqs * 4);
-    // one token per sequence: the cluster kernel that splits the weight stream over 8 SMs per 8 rows
-    // (needs 16-byte loadable weight rows and fits its two row blocks in default shared memory)
+    // one token per sequence: one launch per fully connected layer, features spread over all SMs
+    // (needs 16-byte loadable weight rows and its row block in shared memory)
     const int vl = 16 / c->elem;
-    bool cluster_ok = n_tokens == 1 && (size_t)8 * (c->max_in + c->max_m) * sizeof(float) <= 200 * 1024;
-    for (int w = 0; w < 2 && cluster_ok; ++w) {
+    bool split_ok = n_tokens == 1 && encode_split_smem(c->max_in, c->max_m) <= 200 * 1024;
+    for (int w = 0; w < 2 && split_ok; ++w) {
         const AEHost &ae = c->ae[layer * 2 + w];
-        if (ae.set && (ae.in_dim % vl || ae.hidden % vl)) cluster_ok = false;
+        if (ae.set && (ae.in_dim % vl || ae.hidden % vl)) split_ok = false;
     }
-    cudaError_t e = cluster_ok ? launch_encode_cluster(a, sl, c->cfg.storage, c->max_in, c->max_m, st)
-                               : launch_encode_generic(a, sl, c->cfg.storage, c->max_in, c->max_m, st);
+    const int nb = std::min(c->cfg.max_seqs, KVCAR_MAX_BATCH);
+    cudaError_t e = split_ok ? launch_encode_split(a, sl, c->cfg.storage, c->max_in, c->max_m, c->max_d,
+                                                   reinterpret_cast<float *>(c->ws + c->enchid_off), nb, st)
+                             : launch_encode_generic(a, sl, c->cfg.storage, c->max_in, c->max_m, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "encode launch");
-    ++c->launches;
+    c->launches += split_ok ? 2 : 1;
     return KVCAR_OK;
 }
 

@@ -1,39 +1,45 @@
 // Decode-time encoder + append (one new token per sequence).
 //
 // A batch of B rows meets weights that are far larger than the rows (GPT-2 shape:
-// 0.9 MB per K or V encoder), so the cost is streaming the weights once, and one
-// SM cannot stream them fast enough.  A cluster of 8 CTAs shares each block of 8
-// rows: every CTA computes one eighth of the hidden features (one warp per
-// feature row of FC1, lanes over the input dimension, 16-byte loads), broadcasts
-// its slice of the activated hidden vector into all 8 CTAs' shared memory, and
-// after a cluster barrier computes one eighth of the latent features the same way.
+// 0.9 MB per K or V encoder), so the cost is streaming the weights once, and that
+// needs the whole machine: each of the two fully connected layers is its own launch
+// whose grid spreads the layer's output features over all SMs (one warp per feature:
+// the lanes stream that feature's weight row in 16-byte loads and hold it against a
+// block of up to 16 input rows staged in shared memory).  The hidden activations
+// travel between the two launches through a small fp32 scratch in the workspace.
+// Both launches use programmatic dependent launch: a kernel starts while its
+// predecessor in the stream drains, fetches its first weights, and only then waits
+// for the predecessor's results.
+#include <algorithm>
+
 #include "kvcar_internal.h"
 
 namespace kvcar {
 
 namespace {
 
-constexpr int CR = 8;     // rows per cluster
-constexpr int CSIZE = 8;  // CTAs per cluster
-constexpr int NW = 8;     // warps per CTA
+constexpr int RB = 16;  // input rows per CTA
+constexpr int NW = 8;   // warps (= output features) per CTA
 
 template <typename T>
-struct Ld16;
+struct Vec16;
 template <>
-struct Ld16<float> {
+struct Vec16<float> {
     static constexpr int N = 4;
-    static __device__ __forceinline__ void load(const float *p, float *w) {
-        float4 v = __ldg(reinterpret_cast<const float4 *>(p));
-        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    static __device__ __forceinline__ uint4 load(const float *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
+    static __device__ __forceinline__ void unpack(const uint4 &v, float *w) {
+        w[0] = __uint_as_float(v.x); w[1] = __uint_as_float(v.y); w[2] = __uint_as_float(v.z); w[3] = __uint_as_float(v.w);
     }
     static __device__ __forceinline__ float one(const float *p) { return __ldg(p); }
     static __device__ __forceinline__ void store(float *p, float v) { *p = v; }
 };
 template <>
-struct Ld16<__nv_bfloat16> {
+struct Vec16<__nv_bfloat16> {
     static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float *w) {
-        uint4 v = __ldg(reinterpret_cast<const uint4 *>(p));
+    static __device__ __forceinline__ uint4 load(const __nv_bfloat16 *p) {
+        return __ldg(reinterpret_cast<const uint4 *>(p));
+    }
+    static __device__ __forceinline__ void unpack(const uint4 &v, float *w) {
         const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -45,144 +51,189 @@ struct Ld16<__nv_bfloat16> {
     static __device__ __forceinline__ void store(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
 };
 
-__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// one warp: dot products of weight row `wrow` (length n) with CR activation rows in shared memory
+// acc[r] += sum over this lane's share of w[0..n) * x[r][0..n); `pre` holds the lane's first vector already
 template <typename T>
-__device__ __forceinline__ void warp_dots(const T *wrow, const float *x, int n, int lane, float *acc) {
-    constexpr int VL = Ld16<T>::N;
-#pragma unroll
-    for (int r = 0; r < CR; ++r) acc[r] = 0.f;
+__device__ __forceinline__ void lane_dots(const T *wrow, const uint4 &pre, const float *x, int n, int lane, float *acc) {
+    constexpr int VL = Vec16<T>::N;
+    uint4 cur = pre;
     for (int k0 = lane * VL; k0 < n; k0 += 32 * VL) {
+        const int kn = k0 + 32 * VL;
+        uint4 nxt = cur;
+        if (kn < n) nxt = Vec16<T>::load(wrow + kn);
         float w[VL];
-        Ld16<T>::load(wrow + k0, w);
+        Vec16<T>::unpack(cur, w);
 #pragma unroll
-        for (int r = 0; r < CR; ++r) {
+        for (int r = 0; r < RB; ++r) {
             const float4 *xr = reinterpret_cast<const float4 *>(x + r * n + k0);
 #pragma unroll
             for (int i = 0; i < VL / 4; ++i) {
-                float4 xv = xr[i];
+                const float4 xv = xr[i];
                 acc[r] = fmaf(w[4 * i + 0], xv.x, acc[r]);
                 acc[r] = fmaf(w[4 * i + 1], xv.y, acc[r]);
                 acc[r] = fmaf(w[4 * i + 2], xv.z, acc[r]);
                 acc[r] = fmaf(w[4 * i + 3], xv.w, acc[r]);
             }
         }
-    }
-#pragma unroll
-    for (int r = 0; r < CR; ++r) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
+        cur = nxt;
     }
 }
 
-template <typename T>
-__global__ void __cluster_dims__(CSIZE, 1, 1) __launch_bounds__(NW * 32)
-    encode_cluster_kernel(const __grid_constant__ EncodeArgs a, const __grid_constant__ SeqList seqs) {
-    extern __shared__ __align__(16) float smem[];
-    const int which = blockIdx.y;
-    const EncPlan &pl = a.plan[which];
-    const int rank = blockIdx.x % CSIZE, r0 = (blockIdx.x / CSIZE) * CR;
-    const int n_rows = seqs.n;
-    const int in_dim = pl.in_dim, m = pl.m, d = pl.d;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float *xs = smem;                // [CR][in_dim]
-    float *hs = smem + CR * in_dim;  // [CR][m], filled by all CTAs of the cluster
-    __shared__ int64_t rows[CR];
-    const T *src = reinterpret_cast<const T *>(which == 0 ? a.k : a.v);
-
-    if (threadIdx.x < CR) {
-        const int r = r0 + threadIdx.x;
-        int64_t row = -1;
-        if (r < n_rows) {
-            const int seq = seqs.id[r];
-            const int t = a.seq_len[seq];
-            const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
-            row = (int64_t)page * a.page_tokens + t % a.page_tokens;
-        }
-        rows[threadIdx.x] = row;
+// after the call lane r (r < RB) holds the warp-wide sum of acc[r]
+__device__ __forceinline__ float reduce_rows(float *acc, int lane) {
+    // fold 16 accumulators over 32 lanes: halve the accumulator count while halving the lane distance
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {  // distance 16: lanes < 16 keep rows 0..7, lanes >= 16 keep rows 8..15
+        const float keep = (lane & 16) ? acc[r + 8] : acc[r];
+        const float give = (lane & 16) ? acc[r] : acc[r + 8];
+        acc[r] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
     }
-    if (rank == 0) {  // exact current-token rows (all heads)
-        for (int idx = threadIdx.x; idx < CR * a.kv_width; idx += blockDim.x) {
-            const int rr = idx / a.kv_width, c = idx % a.kv_width, r = r0 + rr;
-            if (r < n_rows)
-                reinterpret_cast<T *>(pl.cur)[(int64_t)seqs.id[r] * a.kv_width + c] = src[(int64_t)r * a.kv_width + c];
-        }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const float keep = (lane & 8) ? acc[r + 4] : acc[r];
+        const float give = (lane & 8) ? acc[r] : acc[r + 4];
+        acc[r] = keep + __shfl_xor_sync(0xffffffffu, give, 8);
     }
-    for (int idx = threadIdx.x; idx < CR * in_dim; idx += blockDim.x) {
-        const int rr = idx / in_dim, c = idx % in_dim, r = r0 + rr;
-        float v = 0.f;
-        if (r < n_rows) v = Ld16<T>::one(src + (int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd);
-        xs[idx] = v;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const float keep = (lane & 4) ? acc[r + 2] : acc[r];
+        const float give = (lane & 4) ? acc[r] : acc[r + 2];
+        acc[r] = keep + __shfl_xor_sync(0xffffffffu, give, 4);
     }
-    __syncthreads();
-    T *pool = reinterpret_cast<T *>(pl.pool);
-    if (!pl.compressed) {  // raw layer: copy (whole cluster takes this branch, nobody waits on anybody)
-        if (rank == 0)
-            for (int idx = threadIdx.x; idx < CR * in_dim; idx += blockDim.x)
-                if (rows[idx / in_dim] >= 0) Ld16<T>::store(pool + rows[idx / in_dim] * pl.width + idx % in_dim, xs[idx]);
-        return;
-    }
-    // every CTA of the cluster is running (its shared memory may be written) past this point
-    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    // ---- FC1 + BatchNorm + LeakyReLU: this CTA's slice of the hidden features ----
     {
-        const int per = (m + CSIZE - 1) / CSIZE;
-        const int j_hi = min(m, (rank + 1) * per);
-        const T *w1 = reinterpret_cast<const T *>(pl.w1r);
-        const int my_row = lane & 7, peer0 = lane >> 3;  // lane -> (row, two of the eight CTAs)
-        for (int j = rank * per + warp; j < j_hi; j += NW) {
-            float acc[CR];
-            warp_dots<T>(w1 + (int64_t)j * in_dim, xs, in_dim, lane, acc);
-            float mine = 0.f;
-#pragma unroll
-            for (int r = 0; r < CR; ++r) mine = (my_row == r) ? acc[r] : mine;
-            float h = fmaf(mine, pl.s1[j], pl.t1[j]);
-            h = h > 0.f ? h : h * pl.slope;
-            const uint32_t local = smem_addr(hs + my_row * m + j);
-#pragma unroll
-            for (int pp = 0; pp < 2; ++pp) {
-                uint32_t remote;
-                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(peer0 + 4 * pp));
-                asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(h) : "memory");
+        const float keep = (lane & 2) ? acc[1] : acc[0];
+        const float give = (lane & 2) ? acc[0] : acc[1];
+        acc[0] = keep + __shfl_xor_sync(0xffffffffu, give, 2);
+    }
+    acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], 1);
+    // lane l now holds row ((l>>4)&1)*8 + ((l>>3)&1)*4 + ((l>>2)&1)*2 + ((l>>1)&1)
+    return acc[0];
+}
+__device__ __forceinline__ int row_of_lane(int lane) {
+    return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+}
+
+// STAGE 1: hidden = LeakyReLU(BN(W1 x + b1)) -> scratch.  STAGE 2: latent = W2 hidden + b2 -> cache rows.
+// grid = (ceil(features / NW), ceil(rows / RB), 2 [K, V]); block = NW warps.
+template <typename T, int STAGE>
+__global__ void __launch_bounds__(NW * 32)
+    encode_fc_kernel(const __grid_constant__ EncodeArgs a, const __grid_constant__ SeqList seqs, float *hid, int hid_pitch,
+                     int max_batch) {
+    extern __shared__ __align__(16) float xs[];  // [RB][n_in]
+    const int which = blockIdx.z;
+    const EncPlan &pl = a.plan[which];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_rows = seqs.n, r0 = blockIdx.y * RB;
+    const int in_dim = pl.in_dim, m = pl.m, d = pl.d;
+    const int n_in = STAGE == 1 ? in_dim : m, n_out = STAGE == 1 ? m : d;
+    const int j = blockIdx.x * NW + warp;  // this warp's output feature
+    const T *src = reinterpret_cast<const T *>(which == 0 ? a.k : a.v);
+    const bool compressed = pl.compressed != 0;
+
+    // weights do not depend on anything earlier in the stream: start fetching them right away
+    const T *wrow = reinterpret_cast<const T *>(STAGE == 1 ? pl.w1r : pl.w2r) + (int64_t)j * n_in;
+    uint4 pre = make_uint4(0, 0, 0, 0);
+    const bool active = compressed && j < n_out;
+    if (active && lane * Vec16<T>::N < n_in) pre = Vec16<T>::load(wrow + lane * Vec16<T>::N);
+    launch_dependents();
+    grid_dependency_wait();  // inputs, page table and (stage 2) the hidden scratch are final from here on
+
+    if (STAGE == 1) {
+        if (blockIdx.x == 0) {  // exact current-token rows (all heads)
+            for (int idx = threadIdx.x; idx < RB * a.kv_width; idx += blockDim.x) {
+                const int rr = idx / a.kv_width, c = idx % a.kv_width, r = r0 + rr;
+                if (r < n_rows)
+                    reinterpret_cast<T *>(pl.cur)[(int64_t)seqs.id[r] * a.kv_width + c] = src[(int64_t)r * a.kv_width + c];
             }
         }
-    }
-    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    // ---- FC2: this CTA's slice of the latent features, rounded and appended ----
-    {
-        const int per = (d + CSIZE - 1) / CSIZE;
-        const int o_hi = min(d, (rank + 1) * per);
-        const T *w2 = reinterpret_cast<const T *>(pl.w2r);
-        for (int o = rank * per + warp; o < o_hi; o += NW) {
-            float acc[CR];
-            warp_dots<T>(w2 + (int64_t)o * m, hs, m, lane, acc);
-            float mine = 0.f;
-#pragma unroll
-            for (int r = 0; r < CR; ++r) mine = (lane == r) ? acc[r] : mine;
-            if (lane < CR && rows[lane] >= 0) Ld16<T>::store(pool + rows[lane] * pl.width + o, mine + pl.b2[o]);
+        if (!compressed) {  // raw layer: copy the stored heads' slices into the cache rows
+            if (blockIdx.x == 0) {
+                T *pool = reinterpret_cast<T *>(pl.pool);
+                for (int idx = threadIdx.x; idx < RB * in_dim; idx += blockDim.x) {
+                    const int rr = idx / in_dim, c = idx % in_dim, r = r0 + rr;
+                    if (r >= n_rows) continue;
+                    const int seq = seqs.id[r], t = a.seq_len[seq];
+                    const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
+                    const int64_t prow = (int64_t)page * a.page_tokens + t % a.page_tokens;
+                    pool[prow * pl.width + c] = src[(int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd];
+                }
+            }
+            return;
+        }
+        if (blockIdx.x * NW >= n_out) return;
+        for (int idx = threadIdx.x; idx < RB * in_dim; idx += blockDim.x) {
+            const int rr = idx / in_dim, c = idx % in_dim, r = r0 + rr;
+            float v = 0.f;
+            if (r < n_rows) v = Vec16<T>::one(src + (int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd);
+            xs[idx] = v;
+        }
+    } else {
+        if (!compressed || blockIdx.x * NW >= n_out) return;
+        const float *h = hid + ((int64_t)which * max_batch + r0) * hid_pitch;
+        for (int idx = threadIdx.x; idx < RB * m; idx += blockDim.x) {
+            const int rr = idx / m, c = idx % m;
+            xs[idx] = (r0 + rr < n_rows) ? h[(int64_t)rr * hid_pitch + c] : 0.f;
         }
     }
+    __syncthreads();
+    if (!active) return;
+    float acc[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) acc[r] = 0.f;
+    lane_dots<T>(wrow, pre, xs, n_in, lane, acc);
+    const float sum = reduce_rows(acc, lane);
+    const int r = r0 + row_of_lane(lane);
+    if ((lane & 1) || r >= n_rows) return;
+    if (STAGE == 1) {
+        float hv = fmaf(sum, pl.s1[j], pl.t1[j]);
+        hv = hv > 0.f ? hv : hv * pl.slope;
+        hid[((int64_t)which * max_batch + r) * hid_pitch + j] = hv;
+    } else {
+        const int seq = seqs.id[r], t = a.seq_len[seq];
+        const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
+        const int64_t prow = (int64_t)page * a.page_tokens + t % a.page_tokens;
+        Vec16<T>::store(reinterpret_cast<T *>(pl.pool) + prow * pl.width + j, sum + pl.b2[j]);
+    }
+}
+
+template <typename T, int STAGE>
+cudaError_t launch_stage(const EncodeArgs &a, const SeqList &seqs, float *hid, int hid_pitch, int max_batch, int n_out_max,
+                         int n_in_max, cudaStream_t st) {
+    const size_t smem = (size_t)RB * n_in_max * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(encode_fc_kernel<T, STAGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((n_out_max + NW - 1) / NW, (seqs.n + RB - 1) / RB, 2);
+    cfg.blockDim = dim3(NW * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, encode_fc_kernel<T, STAGE>, a, seqs, hid, hid_pitch, max_batch);
 }
 
 }  // namespace
 
-cudaError_t launch_encode_cluster(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m,
-                                  cudaStream_t st) {
-    dim3 grid(CSIZE * ((seqs.n + CR - 1) / CR), 2);
-    const size_t smem = (size_t)CR * (max_in + max_m) * sizeof(float);
+size_t encode_split_smem(int max_in, int max_m) { return (size_t)RB * std::max(max_in, max_m) * sizeof(float); }
+
+cudaError_t launch_encode_split(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m, int max_d,
+                                float *hid, int max_batch, cudaStream_t st) {
     cudaError_t e;
+    const int n_hidden = std::max(max_m, NW);  // raw layers still need one block column for the copy
     if (dtype == KVCAR_F32) {
-        e = cudaFuncSetAttribute(encode_cluster_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        encode_cluster_kernel<float><<<grid, NW * 32, smem, st>>>(a, seqs);
+        e = launch_stage<float, 1>(a, seqs, hid, max_m, max_batch, n_hidden, max_in, st);
+        if (e == cudaSuccess && max_m > 0) e = launch_stage<float, 2>(a, seqs, hid, max_m, max_batch, max_d, max_m, st);
     } else {
-        e = cudaFuncSetAttribute(encode_cluster_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem);
-        if (e != cudaSuccess) return e;
-        encode_cluster_kernel<__nv_bfloat16><<<grid, NW * 32, smem, st>>>(a, seqs);
+        e = launch_stage<__nv_bfloat16, 1>(a, seqs, hid, max_m, max_batch, n_hidden, max_in, st);
+        if (e == cudaSuccess && max_m > 0)
+            e = launch_stage<__nv_bfloat16, 2>(a, seqs, hid, max_m, max_batch, max_d, max_m, st);
     }
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace kvcar

@@ -101,9 +101,11 @@ struct TableUpdates {
 cudaError_t launch_table_updates(int32_t *block_table, int32_t *seq_len, const TableUpdates &u, cudaStream_t st);
 cudaError_t launch_encode_generic(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m,
                                   cudaStream_t st);
-// cluster kernel for one new token per sequence (kvcar_encode.cu)
-cudaError_t launch_encode_cluster(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m,
-                                  cudaStream_t st);
+// one new token per sequence, one launch per fully connected layer (kvcar_encode.cu); `hid` is an fp32 scratch of
+// [2][max_batch][max_m] for the hidden activations
+cudaError_t launch_encode_split(const EncodeArgs &a, const SeqList &seqs, int dtype, int max_in, int max_m, int max_d,
+                                float *hid, int max_batch, cudaStream_t st);
+size_t encode_split_smem(int max_in, int max_m);
 cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int dtype, int max_d, int max_m,
                                   int grid_chunks, cudaStream_t st);
 cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, cudaStream_t st);
