@@ -589,7 +589,7 @@ kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seq
     // one token per sequence: one launch per fully connected layer, features spread over all SMs
     // (needs 16-byte loadable weight rows and its row block in shared memory)
     const int vl = 16 / c->elem;
-    bool split_ok = n_tokens == 1 && encode_split_smem(c->max_in, c->max_m) <= 200 * 1024;
+    bool split_ok = n_tokens == 1 && c->cfg.head_dim % vl == 0 && encode_split_smem(c->max_in, c->max_m) <= 200 * 1024;
     for (int w = 0; w < 2 && split_ok; ++w) {
         const AEHost &ae = c->ae[layer * 2 + w];
         if (ae.set && (ae.in_dim % vl || ae.hidden % vl)) split_ok = false;

@@ -133,49 +133,98 @@ __global__ void __launch_bounds__(NW * 32)
     const bool compressed = pl.compressed != 0;
 
     // weights do not depend on anything earlier in the stream: start fetching them right away
+    constexpr int VL = Vec16<T>::N;
     const T *wrow = reinterpret_cast<const T *>(STAGE == 1 ? pl.w1r : pl.w2r) + (int64_t)j * n_in;
     uint4 pre = make_uint4(0, 0, 0, 0);
     const bool active = compressed && j < n_out;
-    if (active && lane * Vec16<T>::N < n_in) pre = Vec16<T>::load(wrow + lane * Vec16<T>::N);
+    float p0 = 0.f, p1 = 0.f;  // stage 1: fused BatchNorm scale, shift; stage 2: bias
+    if (active) {
+        if (lane * VL < n_in) pre = Vec16<T>::load(wrow + lane * VL);
+        if (STAGE == 1) {
+            p0 = pl.s1[j];
+            p1 = pl.t1[j];
+        } else {
+            p0 = pl.b2[j];
+        }
+    }
     launch_dependents();
     grid_dependency_wait();  // inputs, page table and (stage 2) the hidden scratch are final from here on
 
+    const int rows_here = min(RB, n_rows - r0);
+    const int my_row = row_of_lane(lane);
+    int64_t prow = -1;  // stage 2: cache row of the input row this lane will write
+    if (STAGE == 2 && active && !(lane & 1) && my_row < rows_here) {
+        const int seq = seqs.id[r0 + my_row], t = a.seq_len[seq];
+        const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
+        prow = (int64_t)page * a.page_tokens + t % a.page_tokens;
+    }
     if (STAGE == 1) {
+        const int wv = a.kv_width / VL;  // 16-byte vectors per input row (head_dim is a multiple of the vector)
         if (blockIdx.x == 0) {  // exact current-token rows (all heads)
-            for (int idx = threadIdx.x; idx < RB * a.kv_width; idx += blockDim.x) {
-                const int rr = idx / a.kv_width, c = idx % a.kv_width, r = r0 + rr;
-                if (r < n_rows)
-                    reinterpret_cast<T *>(pl.cur)[(int64_t)seqs.id[r] * a.kv_width + c] = src[(int64_t)r * a.kv_width + c];
+            for (int idx = threadIdx.x; idx < rows_here * wv; idx += blockDim.x) {
+                const int rr = idx / wv, cv = idx % wv, r = r0 + rr;
+                reinterpret_cast<uint4 *>(reinterpret_cast<T *>(pl.cur) + (int64_t)seqs.id[r] * a.kv_width)[cv] =
+                    reinterpret_cast<const uint4 *>(src + (int64_t)r * a.kv_width)[cv];
             }
         }
         if (!compressed) {  // raw layer: copy the stored heads' slices into the cache rows
             if (blockIdx.x == 0) {
                 T *pool = reinterpret_cast<T *>(pl.pool);
-                for (int idx = threadIdx.x; idx < RB * in_dim; idx += blockDim.x) {
+                for (int idx = threadIdx.x; idx < rows_here * in_dim; idx += blockDim.x) {
                     const int rr = idx / in_dim, c = idx % in_dim, r = r0 + rr;
-                    if (r >= n_rows) continue;
                     const int seq = seqs.id[r], t = a.seq_len[seq];
                     const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
-                    const int64_t prow = (int64_t)page * a.page_tokens + t % a.page_tokens;
-                    pool[prow * pl.width + c] = src[(int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd];
+                    const int64_t pr = (int64_t)page * a.page_tokens + t % a.page_tokens;
+                    pool[pr * pl.width + c] = src[(int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd];
                 }
             }
             return;
         }
         if (blockIdx.x * NW >= n_out) return;
-        for (int idx = threadIdx.x; idx < RB * in_dim; idx += blockDim.x) {
-            const int rr = idx / in_dim, c = idx % in_dim, r = r0 + rr;
-            float v = 0.f;
-            if (r < n_rows) v = Vec16<T>::one(src + (int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd);
-            xs[idx] = v;
+        // stage the stored heads' slices of this block's rows as fp32, 16 bytes per load, four loads in flight
+        const int nv = in_dim / VL, total = rows_here * nv;
+        for (int base = threadIdx.x; base < total; base += 4 * blockDim.x) {
+            uint4 v[4];
+            int dst[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = base + u * blockDim.x;
+                dst[u] = -1;
+                if (idx < total) {
+                    const int rr = idx / nv, c = (idx % nv) * VL;
+                    v[u] = Vec16<T>::load(src + (int64_t)(r0 + rr) * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd);
+                    dst[u] = rr * in_dim + c;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (dst[u] >= 0) {
+                    float w[VL];
+                    Vec16<T>::unpack(v[u], w);
+#pragma unroll
+                    for (int i = 0; i < VL; i += 4)
+                        *reinterpret_cast<float4 *>(xs + dst[u] + i) = make_float4(w[i], w[i + 1], w[i + 2], w[i + 3]);
+                }
         }
+        for (int idx = rows_here * in_dim + threadIdx.x; idx < RB * in_dim; idx += blockDim.x) xs[idx] = 0.f;
     } else {
         if (!compressed || blockIdx.x * NW >= n_out) return;
         const float *h = hid + ((int64_t)which * max_batch + r0) * hid_pitch;
-        for (int idx = threadIdx.x; idx < RB * m; idx += blockDim.x) {
-            const int rr = idx / m, c = idx % m;
-            xs[idx] = (r0 + rr < n_rows) ? h[(int64_t)rr * hid_pitch + c] : 0.f;
+        const int nv = m / 4, total = rows_here * nv;
+        for (int base = threadIdx.x; base < total; base += 4 * blockDim.x) {
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = base + u * blockDim.x;
+                if (idx < total) v[u] = *reinterpret_cast<const float4 *>(h + (int64_t)(idx / nv) * hid_pitch + (idx % nv) * 4);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = base + u * blockDim.x;
+                if (idx < total) *reinterpret_cast<float4 *>(xs + (idx / nv) * m + (idx % nv) * 4) = v[u];
+            }
         }
+        for (int idx = rows_here * m + threadIdx.x; idx < RB * m; idx += blockDim.x) xs[idx] = 0.f;
     }
     __syncthreads();
     if (!active) return;
@@ -184,17 +233,13 @@ __global__ void __launch_bounds__(NW * 32)
     for (int r = 0; r < RB; ++r) acc[r] = 0.f;
     lane_dots<T>(wrow, pre, xs, n_in, lane, acc);
     const float sum = reduce_rows(acc, lane);
-    const int r = r0 + row_of_lane(lane);
-    if ((lane & 1) || r >= n_rows) return;
+    if ((lane & 1) || my_row >= rows_here) return;
     if (STAGE == 1) {
-        float hv = fmaf(sum, pl.s1[j], pl.t1[j]);
+        float hv = fmaf(sum, p0, p1);
         hv = hv > 0.f ? hv : hv * pl.slope;
-        hid[((int64_t)which * max_batch + r) * hid_pitch + j] = hv;
+        hid[((int64_t)which * max_batch + r0 + my_row) * hid_pitch + j] = hv;
     } else {
-        const int seq = seqs.id[r], t = a.seq_len[seq];
-        const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
-        const int64_t prow = (int64_t)page * a.page_tokens + t % a.page_tokens;
-        Vec16<T>::store(reinterpret_cast<T *>(pl.pool) + prow * pl.width + j, sum + pl.b2[j]);
+        Vec16<T>::store(reinterpret_cast<T *>(pl.pool) + prow * pl.width + j, sum + p0);
     }
 }
 
