@@ -52,7 +52,7 @@ struct kvcar_ctx {
     std::vector<int> width;                 // elements per row
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
     size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
-    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0;  // inside workspace
+    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0;  // inside workspace
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
     std::vector<LayerPlan> plans_host;
@@ -166,6 +166,8 @@ void compute_layout(kvcar_ctx *c) {
     s = align_up(s + (size_t)nb * (2 * W + 2 * g.n_q_heads * g.head_dim) * c->elem + 4 * 256, 256);
     c->enchid_off = s;  // hidden activations between the two decode-time encoder launches
     s = align_up(s + (size_t)2 * nb * c->max_m * sizeof(float), 256);
+    c->kvsplit_off = s;  // probabilities handed from K clusters to V clusters (tensor-core kernel, small grids)
+    s = align_up(s + tc_split_bytes(g), 256);
     c->ws_bytes = s;
 }
 
@@ -479,6 +481,9 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
     // tensor maps and job tables of the tensor-core kernel (fills their regions of the image)
     tc_setup(c->tc, c->cfg, plans, nl, c->weights, c->tmap_off, c->tcpart_off, img.data(),
              (size_t)g.max_pages * g.page_tokens);
+    c->tc.pbuf = reinterpret_cast<float *>(c->ws + c->kvsplit_off);
+    c->tc.pflags = reinterpret_cast<uint32_t *>(c->ws + c->kvsplit_off +
+                                                (size_t)TC_SPLIT_TILES * g.n_q_heads * 132 * sizeof(float));
     memcpy(&img[c->plan_off], plans, (size_t)nl * sizeof(LayerPlan));
 
     std::vector<EncPlan> enc(nl * 2);
@@ -513,6 +518,7 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
 
     cudaError_t e = cudaMemcpyAsync(c->weights, img.data(), img.size(), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->part_off, st);  // tables, lengths, status
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->kvsplit_off, 0, tc_split_bytes(g), st);  // hand-over flags
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(c, e, "upload of packed weights");
     c->bound = true;

@@ -53,12 +53,18 @@ constexpr int MAX_HID_GROUPS = 4;  // hidden chunks of 256 columns
 struct TileIndex {
     int32_t n_tiles;
     uint32_t first[KVCAR_MAX_BATCH + 1];  // first tile of listed sequence i; first[n] = n_tiles
+    int32_t len[KVCAR_MAX_BATCH];         // cached tokens of listed sequence i (the host's copy of the device table)
 };
 
 struct PairLaunch {
     const TcPart *parts;  // this layer's tables for the chosen split: parts[0 .. split-1]
     uint32_t off_hidden, off_ring, off_part, off_fparam, off_q, off_s, off_bar;
     int32_t nslot, max_m, max_in, split, nq_local;
+    // K/V split (small grids): one cluster restores K and publishes the probabilities, another restores V
+    int32_t kv_split;
+    uint32_t epoch;     // value a probability flag takes in this launch
+    float *pbuf;        // [tile][hq][PSTRIDE] probabilities (+ sum at 128) in global memory
+    uint32_t *pflags;   // [tile][hkv]
 };
 
 // ---------------------------------------------------------------------------- PTX helpers
@@ -224,16 +230,16 @@ struct Bars {
     uint32_t hid_ready;    // [MAX_HID_GROUPS] hidden columns written by both CTAs (leader)
     uint32_t p_ready;      // [1] both CTAs' probabilities of all K heads are in place (both CTAs)
     uint32_t afull, aempty;  // [MAX_AUX] hidden slabs lent to the operand ring while they hold no activations
+    uint32_t src_done;     // [2*TC_MAX_SRC] used once each: every product reading source i's activations is done
 };
 constexpr int MAX_AUX = 4 * MAX_HID_GROUPS;
-constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 1 + 2 * MAX_AUX;
+constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 1 + 2 * MAX_AUX + 2 * TC_MAX_SRC;
 
 struct TileInfo {
     int si, chunk, valid;  // listed-sequence index, tile index inside the sequence, valid tokens (0 = no tile)
 };
 
-__device__ __forceinline__ TileInfo locate_tile(const TileIndex &tix, const SeqList &seqs, const int32_t *seq_len,
-                                                int tile, int n_seqs) {
+__device__ __forceinline__ TileInfo locate_tile(const TileIndex &tix, int tile, int n_seqs) {
     TileInfo t{0, 0, 0};
     if (tile >= tix.n_tiles) return t;
     int lo = 0, hi = n_seqs;  // first[lo] <= tile < first[hi]
@@ -243,7 +249,7 @@ __device__ __forceinline__ TileInfo locate_tile(const TileIndex &tix, const SeqL
     }
     t.si = lo;
     t.chunk = tile - (int)tix.first[lo];
-    const int L = seq_len[seqs.id[lo]];
+    const int L = tix.len[lo];
     t.valid = max(0, min(TILE, L - t.chunk * TILE));
     return t;
 }
@@ -267,13 +273,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 
     const uint32_t rank = blockIdx.x & 1u;  // rank in the cluster = which of the pair's two tiles
     const int cid = blockIdx.x >> 1;
-    const int part_i = cid % lay.split, pair = cid / lay.split;
+    const int per_pair = lay.split * (lay.kv_split ? 2 : 1);  // clusters that share one pair of tiles
+    const int sub = cid % per_pair, pair = cid / per_pair;
+    const int part_i = sub % lay.split;
+    // this cluster's share of the work: K only, V only, or K then V
+    const int which_lo = lay.kv_split ? sub / lay.split : 0, which_hi = lay.kv_split ? which_lo + 1 : 2;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hq = a.hq, group = a.hq / a.hkv;
     const bool leader = rank == 0;
 
-    const TileInfo tl[2] = {locate_tile(tix, seqs, a.seq_len, 2 * pair, seqs.n),
-                            locate_tile(tix, seqs, a.seq_len, 2 * pair + 1, seqs.n)};
+    const TileInfo tl[2] = {locate_tile(tix, 2 * pair, seqs.n), locate_tile(tix, 2 * pair + 1, seqs.n)};
     const TileInfo mine = tl[rank];
 
     // carve shared memory (1024-byte aligned for the swizzled tiles; same offsets in both CTAs)
@@ -295,6 +304,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     B.p_ready = B.hid_ready + 8 * MAX_HID_GROUPS;
     B.afull = B.p_ready + 8;
     B.aempty = B.afull + 8 * MAX_AUX;
+    B.src_done = B.aempty + 8 * MAX_AUX;
 
     {  // this cluster's job tables -> shared memory
         const uint4 *src = reinterpret_cast<const uint4 *>(lay.parts + part_i);
@@ -317,6 +327,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             mbar_init(B.afull + 8 * i, 1);
             mbar_init(B.aempty + 8 * i, 1);
         }
+        for (int i = 0; i < 2 * TC_MAX_SRC; ++i) mbar_init(B.src_done + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // tensor memory: all 512 columns in both CTAs of the pair (one CTA per SM by shared memory)
@@ -335,8 +346,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     if (warp == 0 || warp == PRODUCER2_WARP) {
         // ============================== TMA producers (both CTAs) ==============================
         // Two warps share the loads (issuing one tensor load costs its thread ~100 cycles): the loads of the job
-        // list are numbered and producer `pid` issues those of its parity.  Both walk the same places and wait
-        // for each of them to be free, so both see the same ring state.
+        // list are numbered and producer `pid` issues those of its parity.  Both walk the same sequence of
+        // places and keep the same ring state; each waits only for the places it fills.
         const uint32_t pid = warp == 0 ? 0u : 1u;
         if (lane == 0) {
             // pool rows of the tile's two 64-token halves (a half with no valid token re-reads a valid row block)
@@ -353,23 +364,29 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0;
             // wait for the ring slot to be free in this CTA; its owner announces the pair's bytes (leader)
             auto acquire = [&](uint32_t pair_bytes, bool own) -> uint32_t {
-                mbar_wait(B.empty + 8 * slot, phase ^ 1u, a.status, &abort_flag, 0x101);
-                if (own && leader) mbar_expect_tx(B.full + 8 * slot, pair_bytes);
+                if (own) {
+                    mbar_wait(B.empty + 8 * slot, phase ^ 1u, a.status, &abort_flag, 0x101);
+                    if (leader) mbar_expect_tx(B.full + 8 * slot, pair_bytes);
+                }
                 const uint32_t s = slot;
                 if (++slot == (uint32_t)lay.nslot) { slot = 0; phase ^= 1u; }
                 return s;
             };
             // Hidden-chunk jobs also stage operands in the hidden slabs that hold no activations yet (those of
             // this chunk and of later chunks): the ring alone is too shallow for the L2 latency at their rate.
-            // A job takes the ring slots first, so every product that read the previous source's activations
-            // is known to be done (its ring slots have been seen free) before the first slab is overwritten.
             const int ks_hid = (lay.max_m + 63) >> 6;
-            for (int which = 0; which < 2; ++which) {
+            uint32_t n_sources = 0;
+            bool prev_done = true;
+            for (int which = which_lo; which < which_hi; ++which) {
                 const int nj = P.n_jobs[which];
                 for (int j = 0; j < nj; ++j) {
                     const TcJob job = P.jobs[which][j];
                     const TcSrc &sp = P.src[which][job.src];
                     if (job.kind == 1) {
+                        if (job.first) {
+                            ++n_sources;
+                            prev_done = false;
+                        }
                         const int ks1 = (sp.d + 63) >> 6;
                         const int half_rows = job.nc >> 1;  // weight rows this CTA supplies
                         const int y0 = job.c0 + (int)rank * half_rows;
@@ -383,9 +400,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 fb = map_to_cta(B.full + 8 * sl, 0);
                             } else {
                                 const uint32_t x = (uint32_t)(aux_lo + r - lay.nslot);
-                                mbar_wait(B.aempty + 8 * x, ((aux_phase >> x) & 1u) ^ 1u, a.status, &abort_flag, 0x103);
+                                if (own) {
+                                    // nothing reads the previous source's activations any more
+                                    if (n_sources > 1 && !prev_done) {
+                                        mbar_wait(B.src_done + 8 * (n_sources - 2), 0, a.status, &abort_flag, 0x102);
+                                        prev_done = true;
+                                    }
+                                    mbar_wait(B.aempty + 8 * x, ((aux_phase >> x) & 1u) ^ 1u, a.status, &abort_flag, 0x103);
+                                    if (leader) mbar_expect_tx(B.afull + 8 * x, pair_bytes);
+                                }
                                 aux_phase ^= 1u << x;
-                                if (own && leader) mbar_expect_tx(B.afull + 8 * x, pair_bytes);
                                 dst = s_hidden + x * SLOT_BYTES;
                                 fb = map_to_cta(B.afull + 8 * x, 0);
                             }
@@ -440,15 +464,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // The whole warp walks the job list (warp-uniform control flow and operands); one lane issues.
         if (leader) {
             const bool issuer = lane == 0;
-            uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0;
+            uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0, n_done = 0;
             const int ks_hid = (lay.max_m + 63) >> 6;
-            auto wait_full = [&]() -> uint32_t {
-                mbar_wait(B.full + 8 * slot, phase, a.status, &abort_flag, 0x201);
-                const uint32_t s = slot;
+            // A staging place as the consumer sees it.  The poll of the next K slab's barrier is issued before
+            // the current slab's products (its answer takes ~200 cycles to come back under load) and only
+            // turned into a wait afterwards.
+            struct Place { uint32_t addr, fbar, ebar, parity; };
+            auto next_ring = [&]() -> Place {
+                Place pl{s_ring + slot * SLOT_BYTES, B.full + 8 * slot, B.empty + 8 * slot, phase};
                 if (++slot == (uint32_t)lay.nslot) { slot = 0; phase ^= 1u; }
-                return s;
+                return pl;
             };
-            for (int which = 0; which < 2; ++which) {
+            for (int which = which_lo; which < which_hi; ++which) {
                 const int nj = P.n_jobs[which];
                 for (int j = 0; j < nj; ++j, ++jc) {
                     const TcJob job = P.jobs[which][j];
@@ -463,54 +490,85 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         const uint32_t idesc = make_idesc(256, job.nc);
                         const int aux_lo = job.c0 >> 6, n_pool = lay.nslot + (ks_hid - aux_lo);
                         int r = 0;
-                        // next staging place of this job (same order as the producer): smem address, its empty barrier
-                        auto wait_full1 = [&](uint32_t &addr, uint32_t &ebar) {
+                        // next staging place of this job (same order as the producers)
+                        auto next1 = [&]() -> Place {
+                            Place pl;
                             if (r < lay.nslot) {
-                                const uint32_t sl = wait_full();
-                                addr = s_ring + sl * SLOT_BYTES;
-                                ebar = B.empty + 8 * sl;
+                                pl = next_ring();
                             } else {
                                 const uint32_t x = (uint32_t)(aux_lo + r - lay.nslot);
-                                mbar_wait(B.afull + 8 * x, (aux_phase >> x) & 1u, a.status, &abort_flag, 0x205);
+                                pl = Place{s_hidden + x * SLOT_BYTES, B.afull + 8 * x, B.aempty + 8 * x, (aux_phase >> x) & 1u};
                                 aux_phase ^= 1u << x;
-                                addr = s_hidden + x * SLOT_BYTES;
-                                ebar = B.aempty + 8 * x;
                             }
                             if (++r == n_pool) r = 0;
+                            return pl;
                         };
+                        Place z = next1(), w = next1();
+                        mbar_wait(z.fbar, z.parity, a.status, &abort_flag, 0x201);
+                        mbar_wait(w.fbar, w.parity, a.status, &abort_flag, 0x205);
                         for (int ks = 0; ks < ks1; ++ks) {
-                            uint32_t az, ez, aw, ew2;
-                            wait_full1(az, ez);
-                            wait_full1(aw, ew2);
+                            Place zn = z, wn = w;
+                            uint32_t okz = 1, okw = 1;
+                            if (ks + 1 < ks1) {
+                                zn = next1();
+                                wn = next1();
+                                okz = mbar_try<false>(zn.fbar, zn.parity);
+                                okw = mbar_try<false>(wn.fbar, wn.parity);
+                            }
                             tc_fence_after();
                             if (issuer) {
-                                issue_kslab(acc, make_desc(az), make_desc(aw), idesc, min(4, (d - 64 * ks) >> 4), ks == 0);
-                                umma_commit_pair(ez);
-                                umma_commit_pair(ew2);
+                                issue_kslab(acc, make_desc(z.addr), make_desc(w.addr), idesc, min(4, (d - 64 * ks) >> 4),
+                                            ks == 0);
+                                umma_commit_pair(z.ebar);
+                                umma_commit_pair(w.ebar);
                             }
+                            if (!okz) mbar_wait(zn.fbar, zn.parity, a.status, &abort_flag, 0x201);
+                            if (!okw) mbar_wait(wn.fbar, wn.parity, a.status, &abort_flag, 0x205);
+                            z = zn;
+                            w = wn;
                         }
                     } else {
                         const int ks2 = (m + 63) >> 6;
                         const uint32_t idesc = which == 0 ? make_idesc(256, 64 * job.nh) : make_idesc(256, 256);
                         const bool first_use = job.first != 0;  // first head group of this source
+                        Place w = next_ring();
+                        if (first_use) {
+                            mbar_wait(B.hid_ready, hid_phase & 1u, a.status, &abort_flag, 0x204);
+                            hid_phase ^= 1u;
+                        }
+                        mbar_wait(w.fbar, w.parity, a.status, &abort_flag, 0x201);
                         for (int ks = 0; ks < ks2; ++ks) {
-                            if (first_use && (ks & 3) == 0) {
-                                const int g = ks >> 2;
-                                mbar_wait(B.hid_ready + 8 * g, (hid_phase >> g) & 1u, a.status, &abort_flag, 0x204);
-                                hid_phase ^= 1u << g;
+                            Place wn = w;
+                            uint32_t okw = 1;
+                            if (ks + 1 < ks2) {
+                                wn = next_ring();
+                                okw = mbar_try<false>(wn.fbar, wn.parity);
                             }
-                            const uint32_t sw = wait_full();
                             tc_fence_after();
                             const uint64_t dh = make_desc(s_hidden + ks * SLOT_BYTES);
-                            const uint64_t dw = make_desc(s_ring + sw * SLOT_BYTES);
+                            const uint64_t dw = make_desc(w.addr);
                             const int nk = min(4, (m - 64 * ks) >> 4);
                             if (issuer) {
                                 if (which == 0)
                                     issue_kslab(acc, dh, dw, idesc, nk, ks == 0);
                                 else
                                     issue_kslab(acc, dw, dh, idesc, nk, ks == 0);
-                                umma_commit_pair(B.empty + 8 * sw);
+                                umma_commit_pair(w.ebar);
                             }
+                            if (ks + 1 < ks2) {
+                                if (first_use && ((ks + 1) & 3) == 0) {  // the next slab starts a new hidden chunk
+                                    const int g = (ks + 1) >> 2;
+                                    mbar_wait(B.hid_ready + 8 * g, (hid_phase >> g) & 1u, a.status, &abort_flag, 0x204);
+                                    hid_phase ^= 1u << g;
+                                }
+                                if (!okw) mbar_wait(wn.fbar, wn.parity, a.status, &abort_flag, 0x201);
+                            }
+                            w = wn;
+                        }
+                        // last head group of this source: its hidden slabs may be lent to the ring again
+                        if (j + 1 == nj || P.jobs[which][j + 1].kind == 1) {
+                            if (issuer) umma_commit_pair(B.src_done + 8 * n_done);
+                            ++n_done;
                         }
                     }
                     if (issuer) umma_commit_pair(B.jfull + 8 * buf);
@@ -536,7 +594,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         if (mine.valid > 0) {
             // pull this tile's latent rows of every source from HBM into L2 ahead of the producers' loads
             int item = 0;
-            for (int which = 0; which < 2; ++which)
+            for (int which = which_lo; which < which_hi; ++which)
                 for (int sidx = 0; sidx < P.n_src[which]; ++sidx) {
                     const TcSrc &sp = P.src[which][sidx];
                     const int n = 2 * ((sp.d + 63) >> 6);
@@ -555,9 +613,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             for (int i = et; i < nq_part * 64; i += 256) qs[i] = __bfloat162float(qg[i]) * a.scale;
         }
         uint32_t jc = 0;
-        for (int which = 0; which < 2; ++which) {
+        for (int which = which_lo; which < which_hi; ++which) {
             const int nj = P.n_jobs[which];
-            if (which == 1) {
+            if (which == 1 && !lay.kv_split) {
                 // every probability this CTA will read has been written, here and by the peer
                 asm volatile("fence.acq_rel.cluster;" ::: "memory");
                 __syncwarp();
@@ -637,6 +695,40 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     continue;
                 }
                 // ---- head group ----
+                if (which == 1 && lay.kv_split) {
+                    // fetch the probabilities of this job's heads, both tiles, from the K cluster (global memory):
+                    // wait for each row's flag, copy the row into this CTA's buffer
+                    const int rows_per_tile = 4 * group, n_vec = 2 * rows_per_tile * (PSTRIDE / 4);
+                    for (int idx = et; idx < n_vec; idx += 256) {
+                        const int rrow = idx / (PSTRIDE / 4), v4 = idx % (PSTRIDE / 4);
+                        const int th = rrow / rows_per_tile, hp = (rrow % rows_per_tile) / group, g = rrow % group;
+                        const int kvh = job.kvh[hp];
+                        if (kvh < 0 || tl[th].valid == 0) continue;
+                        const int tile = 2 * pair + th;
+                        const uint32_t *fl = lay.pflags + (size_t)tile * a.hkv + kvh;
+                        uint32_t seen = 0, n = 0;
+                        uint64_t t0 = 0;
+                        while (true) {
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(fl) : "memory");
+                            if (seen == lay.epoch) break;
+                            __nanosleep(200);
+                            if ((++n & 63u) == 0) {  // bounded like every other wait of this kernel
+                                const uint64_t now = global_ns();
+                                if (t0 == 0) t0 = now;
+                                if (now - t0 > (abort_flag ? 2000000ull : 2000000000ull)) {
+                                    abort_flag = 1;
+                                    atomicCAS(a.status, 0, 0x304);
+                                    break;
+                                }
+                            }
+                        }
+                        const int ql = (kvh - h_lo) * group + g;
+                        const float4 val = __ldcg(reinterpret_cast<const float4 *>(
+                                                      lay.pbuf + ((size_t)tile * hq + h_lo * group + ql) * PSTRIDE) + v4);
+                        *reinterpret_cast<float4 *>(Sall + ((size_t)th * lay.nq_local + ql) * PSTRIDE + 4 * v4) = val;
+                    }
+                    epi_bar_sync();
+                }
                 mbar_wait<false, 100>(B.jfull + 8 * buf, (jc >> 1) & 1u, a.status, &abort_flag, 0x302);
                 tc_fence_after();
                 if (which == 0) {
@@ -689,12 +781,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
                             *reinterpret_cast<float4 *>(srow + 4 * lane) = sc;
-                            const uint32_t prow = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE) * 4u;
-                            st_cluster_v4(prow + 16u * lane, sc.x, sc.y, sc.z, sc.w);
+                            const int qh = h_lo * group + ql;
+                            if (lay.kv_split) {
+                                float *grow = lay.pbuf + ((size_t)(2 * pair + (int)rank) * hq + qh) * PSTRIDE;
+                                *reinterpret_cast<float4 *>(grow + 4 * lane) = sc;
+                                if (lane == 0) grow[128] = sum;
+                            } else {
+                                const uint32_t prow = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE) * 4u;
+                                st_cluster_v4(prow + 16u * lane, sc.x, sc.y, sc.z, sc.w);
+                                if (lane == 0) st_cluster_f32(prow + 128u * 4u, sum);
+                            }
                             if (lane == 0) {
                                 srow[128] = sum;
-                                st_cluster_f32(prow + 128u * 4u, sum);
-                                const int qh = h_lo * group + ql;
                                 float *part =
                                     a.partials + (((int64_t)mine.si * a.max_chunks + mine.chunk) * hq + qh) * (64 + 2);
                                 part[0] = mx;
@@ -702,9 +800,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             }
                         }
                     }
+                    if (lay.kv_split) {
+                        // publish: this job's heads of this tile are in global memory for the V cluster
+                        __threadfence();
+                        epi_bar_sync();
+                        if (et < nh && mine.valid > 0)
+                            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(lay.pflags + (size_t)(2 * pair + (int)rank) *
+                                                                                        a.hkv + job.kvh[et]),
+                                         "r"(lay.epoch)
+                                         : "memory");
+                    }
                 } else {
                     // V: this thread owns (head place, channel) = row; columns = tokens of tile chalf
-                    if (!p_waited) {
+                    if (!lay.kv_split && !p_waited) {
                         mbar_wait<true, 100>(B.p_ready, 0, a.status, &abort_flag, 0x303);
                         p_waited = true;
                     }
@@ -901,6 +1009,9 @@ inline int part_index(int split, int i) { return (split == 1 ? 0 : split == 2 ? 
 }  // namespace
 
 size_t tc_part_bytes(int n_layers) { return (size_t)n_layers * 7 * sizeof(TcPart); }
+size_t tc_split_bytes(const kvcar_config &cfg) {
+    return (size_t)TC_SPLIT_TILES * ((size_t)cfg.n_q_heads * PSTRIDE * sizeof(float) + (size_t)cfg.n_kv_heads * sizeof(uint32_t));
+}
 
 void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int n_layers, char *weights_dev,
               size_t tmap_off, size_t part_off, char *img, size_t pool_rows) {
@@ -1004,27 +1115,41 @@ bool tc_layer_supported(const TcState &tc, int layer) {
     return tc.available && layer >= 0 && layer < TC_MAX_LAYERS && tc.layer[layer].ok;
 }
 
-cudaError_t tc_launch_decode(const TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
+cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
                              int layer, cudaStream_t st) {
     const TcLayerCfg &lc = tc.layer[layer];
     TileIndex tix;
     uint32_t t = 0;
     for (int i = 0; i < seqs.n; ++i) {
         tix.first[i] = t;
+        tix.len[i] = lens[i];
         t += (uint32_t)((lens[i] + TILE - 1) / TILE);
     }
     tix.first[seqs.n] = t;
     tix.n_tiles = (int32_t)t;
     if (t == 0) return cudaSuccess;
     const int n_pairs = (int)((t + 1) / 2);
-    // small grids: split the KV heads over more clusters while everything still runs in one wave
-    int split = 1;
-    if (lc.split_ok[2] && 2 * n_pairs * 4 <= tc.n_sms) split = 4;
-    else if (lc.split_ok[1] && 2 * n_pairs * 2 <= tc.n_sms) split = 2;
+    // Small grids: spread the work of a tile pair over more clusters while everything still runs in one wave.
+    // First K and V go to separate clusters (nothing is computed twice: the probabilities cross through global
+    // memory, which needs both clusters on the machine at once - true below the SM count); then the KV heads
+    // are split (each cluster repeats the hidden layer for its heads).
+    int split = 1, kv_split = 0;
+    if (tc.pbuf && 4 * n_pairs <= tc.n_sms) {
+        kv_split = 1;
+        if (lc.split_ok[1] && 8 * n_pairs <= tc.n_sms) split = 2;
+    } else if (lc.split_ok[2] && 2 * n_pairs * 4 <= tc.n_sms) {
+        split = 4;
+    } else if (lc.split_ok[1] && 2 * n_pairs * 2 <= tc.n_sms) {
+        split = 2;
+    }
     const int group = a.hq / a.hkv;
     const int nq_local = a.hkv / split * group;
     PairLaunch lay = make_launch(nq_local, lc.max_m, lc.max_in, pick_nslot(nq_local, lc.max_m, lc.max_in));
     lay.split = split;
+    lay.kv_split = kv_split;
+    lay.epoch = ++tc.epoch;
+    lay.pbuf = tc.pbuf;
+    lay.pflags = tc.pflags;
     lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * 7 + part_index(split, 0);
     // never less than half an SM's shared memory: two CTAs on one SM would both want all of tensor memory
     const int smem = (int)std::max(launch_bytes(lay), 120u * 1024u);
@@ -1034,7 +1159,7 @@ cudaError_t tc_launch_decode(const TcState &tc, const DecodeArgs &a, const SeqLi
         if (e != cudaSuccess) return e;
         configured_smem = smem;
     }
-    dim3 grid(2 * n_pairs * split);
+    dim3 grid(2 * n_pairs * split * (kv_split ? 2 : 1));
     decode_pair_kernel<<<grid, NTHREADS, smem, st>>>(a, seqs, tix, lay);
     return cudaGetLastError();
 }

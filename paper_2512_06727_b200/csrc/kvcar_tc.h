@@ -7,6 +7,7 @@ namespace kvcar {
 constexpr int TC_MAX_LAYERS = 512;
 constexpr int TC_MAX_SRC = 6;    // distinct source layers per K or V of one head subset
 constexpr int TC_MAX_JOBS = 24;  // accumulator jobs per K or V of one head subset
+constexpr int TC_SPLIT_TILES = 160;  // the K/V split is used only while 2 x tiles <= SM count
 constexpr int TC_MAX_SPLIT = 4;  // a layer's KV heads can be split over up to 4 clusters per tile pair
 
 // One source layer as the tensor-core kernel sees it.
@@ -53,11 +54,17 @@ struct TcState {
     const char *why = "not set up";
     char *parts_dev = nullptr;  // TcPart[n_layers][7] in the weights buffer: split 1 -> [0], 2 -> [1..2], 4 -> [3..6]
     int n_sms = 148;
+    // K/V split of small grids: probabilities cross from the K cluster to the V cluster through these
+    float *pbuf = nullptr;       // [TC_SPLIT_TILES][n_q_heads][132]
+    uint32_t *pflags = nullptr;  // [TC_SPLIT_TILES][n_kv_heads], zero at bind time
+    uint32_t epoch = 0;          // launches so far; a flag equal to it belongs to the current launch
     TcLayerCfg layer[TC_MAX_LAYERS];
 };
 
 // bytes of the per-layer job tables inside the weights buffer
 size_t tc_part_bytes(int n_layers);
+// bytes of the probability hand-over area (pbuf then pflags) inside the workspace
+size_t tc_split_bytes(const kvcar_config &cfg);
 
 // Build the TMA descriptors and the per-layer job tables into the host image of the
 // weights buffer (at tmap_off / part_off) and decide per layer whether the tensor-core
@@ -68,7 +75,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans_host,
 void tc_destroy(TcState &tc);
 bool tc_layer_supported(const TcState &tc, int layer);
 // lens: host copy of the listed sequences' lengths (same values the device table holds)
-cudaError_t tc_launch_decode(const TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
+cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
                              int layer, cudaStream_t st);
 
 }  // namespace kvcar

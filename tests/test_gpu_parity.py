@@ -173,6 +173,20 @@ def test_physical_page_permutation_is_bit_invariant(kernel):
         assert np.array_equal(a[l], b[l])
 
 
+def test_large_grid_runs_k_then_v_in_one_cluster():
+    """More tile pairs than a quarter of the SMs: the tensor-core kernel stops spreading a
+    pair over several clusters and each cluster restores K, then V (the other tests are
+    small enough to take the split paths)."""
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=5, cached_tokens=0, decode_steps=1, reuse_frac=0.25)
+    pps = 34
+    p = Pair(w, max_seqs=5, max_pages=5 * pps, max_pages_per_seq=pps, kernel=B.KERNEL_TENSOR)
+    seqs = [0, 1, 2, 3, 4]
+    p.open(seqs)
+    for s_, n in zip(seqs, (2100, 2049, 2111, 2050, 2064)):     # 17 tiles each: 85 tiles, 43 pairs
+        p.prefill([s_], n)
+    _check_step(p.decode_step(seqs, 0), "bf16", "fused clusters")
+
+
 def test_fp32_stack_with_reuse_generic():
     """fp32 mode on a multi-layer stack with chains of reuse; 1e-4 absolute."""
     w = synth.scaled(synth.CONFIGS["c2"], n_layers=4, batch=2, storage="f32", reuse_frac=0.5)
