@@ -748,17 +748,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             y2[2 * c + 1] = __fadd2_rn(make_float2(y[4 * c + 2], y[4 * c + 3]), make_float2(b4.z, b4.w));
                         }
                         const int ql0 = (job.kvh[hp] - h_lo) * group;
-                        for (int g = 0; g < group; ++g) {
-                            const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g) * 64);
-                            float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
+                        // four query heads of the group at a time: eight independent accumulation chains
+                        for (int g0 = 0; g0 < group; g0 += 4) {
+                            float2 d0[4], d1[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) d0[u] = d1[u] = make_float2(0.f, 0.f);
+                            const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g0) * 64);
 #pragma unroll
                             for (int c = 0; c < 16; ++c) {
-                                const float4 qq = q4[c];
-                                d0 = __ffma2_rn(y2[2 * c], make_float2(qq.x, qq.y), d0);
-                                d1 = __ffma2_rn(y2[2 * c + 1], make_float2(qq.z, qq.w), d1);
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    if (g0 + u < group) {
+                                        const float4 qq = q4[16 * u + c];
+                                        d0[u] = __ffma2_rn(y2[2 * c], make_float2(qq.x, qq.y), d0[u]);
+                                        d1[u] = __ffma2_rn(y2[2 * c + 1], make_float2(qq.z, qq.w), d1[u]);
+                                    }
+                                }
                             }
-                            const float dot = (d0.x + d0.y) + (d1.x + d1.y);
-                            Smine[(ql0 + g) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                if (g0 + u < group) {
+                                    const float dot = (d0[u].x + d0[u].y) + (d1[u].x + d1[u].y);
+                                    Smine[(ql0 + g0 + u) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
+                                }
+                            }
                         }
                     }
                     tc_fence_before();
@@ -822,9 +835,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     if (kvh >= 0 && tt.valid > 0) {
                         const int ql0 = (kvh - h_lo) * group;
                         const float *Sp = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE;
-                        float2 accv[8];
+                        float2 accv[8], accw[8];
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) accv[g] = make_float2(0.f, 0.f);
+                        for (int g = 0; g < 8; ++g) accv[g] = accw[g] = make_float2(0.f, 0.f);
                         for (int gi = 0; gi < 4; ++gi) {
                             if (32 * gi >= tt.valid) break;
                             float y[32];
@@ -834,18 +847,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 #pragma unroll
                                 for (int t = 0; t < 32; ++t) y[t] = (32 * gi + t < tt.valid) ? y[t] : 0.f;
                             }
+                            // token groups outside, query heads inside: one accumulation chain per head
 #pragma unroll
-                            for (int g = 0; g < 8; ++g) {
-                                if (g < group) {
-                                    const float4 *p4 = reinterpret_cast<const float4 *>(Sp + g * PSTRIDE + 32 * gi);
-                                    float2 s0 = accv[g], s1v = make_float2(0.f, 0.f);
+                            for (int t = 0; t < 8; ++t) {
+                                const float2 ya = make_float2(y[4 * t], y[4 * t + 1]);
+                                const float2 yb = make_float2(y[4 * t + 2], y[4 * t + 3]);
 #pragma unroll
-                                    for (int t = 0; t < 8; ++t) {
-                                        const float4 pp = p4[t];
-                                        s0 = __ffma2_rn(make_float2(pp.x, pp.y), make_float2(y[4 * t], y[4 * t + 1]), s0);
-                                        s1v = __ffma2_rn(make_float2(pp.z, pp.w), make_float2(y[4 * t + 2], y[4 * t + 3]), s1v);
+                                for (int g = 0; g < 8; ++g) {
+                                    if (g < group) {
+                                        const float4 pp =
+                                            *reinterpret_cast<const float4 *>(Sp + g * PSTRIDE + 32 * gi + 4 * t);
+                                        accv[g] = __ffma2_rn(make_float2(pp.x, pp.y), ya, accv[g]);
+                                        accw[g] = __ffma2_rn(make_float2(pp.z, pp.w), yb, accw[g]);
                                     }
-                                    accv[g] = __fadd2_rn(s0, s1v);
                                 }
                             }
                         }
@@ -855,7 +869,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             if (g < group) {
                                 const int qh = (h_lo * group) + ql0 + g;
                                 float *part = a.partials + (((int64_t)tt.si * a.max_chunks + tt.chunk) * hq + qh) * (64 + 2);
-                                part[2 + c] = (accv[g].x + accv[g].y) + bias * Sp[g * PSTRIDE + 128];
+                                part[2 + c] = ((accv[g].x + accv[g].y) + (accw[g].x + accw[g].y)) + bias * Sp[g * PSTRIDE + 128];
                             }
                         }
                     }
