@@ -56,7 +56,9 @@ typedef enum { KVCAR_K = 0, KVCAR_V = 1 } kvcar_which;
 typedef enum {
     KVCAR_KERNEL_AUTO = 0,    /* tensor-core kernel where the shape allows, else generic */
     KVCAR_KERNEL_GENERIC = 1, /* fp32-FMA kernels (any supported shape, both dtypes)     */
-    KVCAR_KERNEL_TENSOR = 2   /* tcgen05/TMEM fused kernel (bf16 storage only)           */
+    KVCAR_KERNEL_TENSOR = 2,  /* tcgen05/TMEM fused kernel (bf16 storage only)           */
+    KVCAR_KERNEL_RAW = 3      /* reported only: streaming kernel AUTO picks for a layer
+                                 whose K and V are all stored raw (no autoencoder)       */
 } kvcar_kernel;
 
 /* flags of kvcar_decode_attention */
@@ -261,7 +263,7 @@ kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *ctx, double *compressed, dou
 kvcar_status kvcar_layer_work_per_token(kvcar_ctx *ctx, int32_t layer, double *bytes, double *flops);
 /* Number of kernels the library has launched so far on this context. */
 kvcar_status kvcar_launch_count(kvcar_ctx *ctx, int64_t *count);
-/* Kernel family (kvcar_kernel: GENERIC or TENSOR) that kvcar_decode_attention will use
+/* Kernel family (kvcar_kernel: GENERIC, TENSOR or RAW) that kvcar_decode_attention will use
  * for `layer` under the current kvcar_set_kernel choice.  Only after kvcar_bind_memory. */
 kvcar_status kvcar_layer_kernel(kvcar_ctx *ctx, int32_t layer, int32_t *kernel);
 /* Synchronise `stream` and report any asynchronous CUDA error or device-side

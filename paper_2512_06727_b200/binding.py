@@ -16,7 +16,7 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 K, V = 0, 1
-KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TENSOR = 0, 1, 2
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TENSOR, KERNEL_RAW = 0, 1, 2, 3
 INCLUDE_CURRENT_EXACT = 1
 MAX_BATCH = 512
 

@@ -264,6 +264,16 @@ kvcar_status flush_tables(kvcar_ctx *c, cudaStream_t st) {
     return KVCAR_OK;
 }
 
+// every K and V head of the layer reads raw rows, and the shape fits the streaming kernel
+bool layer_is_raw(const kvcar_ctx *c, int layer) {
+    if (c->cfg.head_dim != 64 || c->cfg.n_q_heads / c->cfg.n_kv_heads > 8) return false;
+    const LayerPlan &lp = c->plans_host[layer];
+    for (int w = 0; w < 2; ++w)
+        for (int s = 0; s < lp.w[w].n_src; ++s)
+            if (lp.w[w].src[s].compressed) return false;
+    return true;
+}
+
 bool use_tensor_kernel(const kvcar_ctx *c) {
     if (c->kernel == KVCAR_KERNEL_GENERIC) return false;
     return c->tc.available;
@@ -665,7 +675,9 @@ kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *
         if (c->kernel == KVCAR_KERNEL_TENSOR && !want_tc)
             return fail(c, KVCAR_ERR_UNSUPPORTED, std::string("tensor-core kernel cannot run this layer: ") + c->tc.why);
         cudaError_t e;
-        if (want_tc) {
+        if (c->kernel != KVCAR_KERNEL_GENERIC && layer_is_raw(c, layer)) {
+            e = launch_decode_raw(a, sl, g.storage, n_chunks, st);
+        } else if (want_tc) {
             int32_t lens[KVCAR_MAX_BATCH];
             for (int i = 0; i < n_seqs; ++i) lens[i] = c->len[seqs[i]];
             e = tc_launch_decode(c->tc, a, sl, lens, layer, st);
@@ -792,7 +804,10 @@ kvcar_status kvcar_launch_count(kvcar_ctx *c, int64_t *count) {
 kvcar_status kvcar_layer_kernel(kvcar_ctx *c, int32_t layer, int32_t *kernel) {
     if (!c || !kernel || layer < 0 || layer >= c->cfg.n_layers) return fail(c, KVCAR_ERR_INVALID_ARG, "bad argument");
     if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
-    *kernel = (use_tensor_kernel(c) && tc_layer_supported(c->tc, layer)) ? KVCAR_KERNEL_TENSOR : KVCAR_KERNEL_GENERIC;
+    if (c->kernel != KVCAR_KERNEL_GENERIC && layer_is_raw(c, layer))
+        *kernel = KVCAR_KERNEL_RAW;
+    else
+        *kernel = (use_tensor_kernel(c) && tc_layer_supported(c->tc, layer)) ? KVCAR_KERNEL_TENSOR : KVCAR_KERNEL_GENERIC;
     return KVCAR_OK;
 }
 

@@ -108,6 +108,8 @@ cudaError_t launch_encode_split(const EncodeArgs &a, const SeqList &seqs, int dt
 size_t encode_split_smem(int max_in, int max_m);
 cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int dtype, int max_d, int max_m,
                                   int grid_chunks, cudaStream_t st);
+// raw K/V layers (no autoencoder), head_dim 64, <= 8 query heads per KV head (kvcar_raw.cu)
+cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtype, int grid_chunks, cudaStream_t st);
 cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, cudaStream_t st);
 size_t decode_generic_smem(int hq, int hd, int max_d, int max_m);
 
