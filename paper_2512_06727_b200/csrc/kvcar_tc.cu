@@ -748,30 +748,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             y2[2 * c + 1] = __fadd2_rn(make_float2(y[4 * c + 2], y[4 * c + 3]), make_float2(b4.z, b4.w));
                         }
                         const int ql0 = (job.kvh[hp] - h_lo) * group;
-                        // four query heads of the group at a time: eight independent accumulation chains
-                        for (int g0 = 0; g0 < group; g0 += 4) {
-                            float2 d0[4], d1[4];
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) d0[u] = d1[u] = make_float2(0.f, 0.f);
-                            const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g0) * 64);
+                        for (int g = 0; g < group; ++g) {
+                            const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g) * 64);
+                            float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
 #pragma unroll
                             for (int c = 0; c < 16; ++c) {
-#pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    if (g0 + u < group) {
-                                        const float4 qq = q4[16 * u + c];
-                                        d0[u] = __ffma2_rn(y2[2 * c], make_float2(qq.x, qq.y), d0[u]);
-                                        d1[u] = __ffma2_rn(y2[2 * c + 1], make_float2(qq.z, qq.w), d1[u]);
-                                    }
-                                }
+                                const float4 qq = q4[c];
+                                d0 = __ffma2_rn(y2[2 * c], make_float2(qq.x, qq.y), d0);
+                                d1 = __ffma2_rn(y2[2 * c + 1], make_float2(qq.z, qq.w), d1);
                             }
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                if (g0 + u < group) {
-                                    const float dot = (d0[u].x + d0[u].y) + (d1[u].x + d1[u].y);
-                                    Smine[(ql0 + g0 + u) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
-                                }
-                            }
+                            const float dot = (d0.x + d0.y) + (d1.x + d1.y);
+                            Smine[(ql0 + g) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
                         }
                     }
                     tc_fence_before();
