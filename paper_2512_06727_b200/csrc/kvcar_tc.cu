@@ -230,10 +230,9 @@ struct Bars {
     uint32_t hid_ready;    // [MAX_HID_GROUPS] hidden columns written by both CTAs (leader)
     uint32_t p_ready;      // [1] both CTAs' probabilities of all K heads are in place (both CTAs)
     uint32_t afull, aempty;  // [MAX_AUX] hidden slabs lent to the operand ring while they hold no activations
-    uint32_t src_done;     // [2*TC_MAX_SRC] used once each: every product reading source i's activations is done
 };
 constexpr int MAX_AUX = 4 * MAX_HID_GROUPS;
-constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 1 + 2 * MAX_AUX + 2 * TC_MAX_SRC;
+constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 1 + 2 * MAX_AUX;
 
 struct TileInfo {
     int si, chunk, valid;  // listed-sequence index, tile index inside the sequence, valid tokens (0 = no tile)
@@ -304,7 +303,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     B.p_ready = B.hid_ready + 8 * MAX_HID_GROUPS;
     B.afull = B.p_ready + 8;
     B.aempty = B.afull + 8 * MAX_AUX;
-    B.src_done = B.aempty + 8 * MAX_AUX;
 
     {  // this cluster's job tables -> shared memory
         const uint4 *src = reinterpret_cast<const uint4 *>(lay.parts + part_i);
@@ -327,7 +325,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             mbar_init(B.afull + 8 * i, 1);
             mbar_init(B.aempty + 8 * i, 1);
         }
-        for (int i = 0; i < 2 * TC_MAX_SRC; ++i) mbar_init(B.src_done + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // tensor memory: all 512 columns in both CTAs of the pair (one CTA per SM by shared memory)
@@ -347,7 +344,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // ============================== TMA producers (both CTAs) ==============================
         // Two warps share the loads (issuing one tensor load costs its thread ~100 cycles): the loads of the job
         // list are numbered and producer `pid` issues those of its parity.  Both walk the same sequence of
-        // places and keep the same ring state; each waits only for the places it fills.
+        // places and wait for each of them to be free, so both see the same ring state.
         const uint32_t pid = warp == 0 ? 0u : 1u;
         if (lane == 0) {
             // pool rows of the tile's two 64-token halves (a half with no valid token re-reads a valid row block)
@@ -364,29 +361,25 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0;
             // wait for the ring slot to be free in this CTA; its owner announces the pair's bytes (leader)
             auto acquire = [&](uint32_t pair_bytes, bool own) -> uint32_t {
-                if (own) {
-                    mbar_wait(B.empty + 8 * slot, phase ^ 1u, a.status, &abort_flag, 0x101);
-                    if (leader) mbar_expect_tx(B.full + 8 * slot, pair_bytes);
-                }
+                mbar_wait(B.empty + 8 * slot, phase ^ 1u, a.status, &abort_flag, 0x101);
+                if (own && leader) mbar_expect_tx(B.full + 8 * slot, pair_bytes);
                 const uint32_t s = slot;
                 if (++slot == (uint32_t)lay.nslot) { slot = 0; phase ^= 1u; }
                 return s;
             };
             // Hidden-chunk jobs also stage operands in the hidden slabs that hold no activations yet (those of
             // this chunk and of later chunks): the ring alone is too shallow for the L2 latency at their rate.
+            // A job takes the ring slots first and both producers wait for every place, so every product that
+            // read the previous source's activations is known to be done (its ring slots have been seen free:
+            // completions arrive in issue order) before the first hidden slab is overwritten.
             const int ks_hid = (lay.max_m + 63) >> 6;
-            uint32_t n_sources = 0;
-            bool prev_done = true;
-            for (int which = which_lo; which < which_hi; ++which) {
+            for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
+                if (which < which_lo || which >= which_hi) continue;
                 const int nj = P.n_jobs[which];
                 for (int j = 0; j < nj; ++j) {
                     const TcJob job = P.jobs[which][j];
                     const TcSrc &sp = P.src[which][job.src];
                     if (job.kind == 1) {
-                        if (job.first) {
-                            ++n_sources;
-                            prev_done = false;
-                        }
                         const int ks1 = (sp.d + 63) >> 6;
                         const int half_rows = job.nc >> 1;  // weight rows this CTA supplies
                         const int y0 = job.c0 + (int)rank * half_rows;
@@ -400,15 +393,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 fb = map_to_cta(B.full + 8 * sl, 0);
                             } else {
                                 const uint32_t x = (uint32_t)(aux_lo + r - lay.nslot);
-                                if (own) {
-                                    // nothing reads the previous source's activations any more
-                                    if (n_sources > 1 && !prev_done) {
-                                        mbar_wait(B.src_done + 8 * (n_sources - 2), 0, a.status, &abort_flag, 0x102);
-                                        prev_done = true;
-                                    }
-                                    mbar_wait(B.aempty + 8 * x, ((aux_phase >> x) & 1u) ^ 1u, a.status, &abort_flag, 0x103);
-                                    if (leader) mbar_expect_tx(B.afull + 8 * x, pair_bytes);
-                                }
+                                mbar_wait(B.aempty + 8 * x, ((aux_phase >> x) & 1u) ^ 1u, a.status, &abort_flag, 0x103);
+                                if (own && leader) mbar_expect_tx(B.afull + 8 * x, pair_bytes);
                                 aux_phase ^= 1u << x;
                                 dst = s_hidden + x * SLOT_BYTES;
                                 fb = map_to_cta(B.afull + 8 * x, 0);
@@ -464,18 +450,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // The whole warp walks the job list (warp-uniform control flow and operands); one lane issues.
         if (leader) {
             const bool issuer = lane == 0;
-            uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0, n_done = 0;
+            uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0;
             const int ks_hid = (lay.max_m + 63) >> 6;
-            // A staging place as the consumer sees it.  The poll of the next K slab's barrier is issued before
-            // the current slab's products (its answer takes ~200 cycles to come back under load) and only
-            // turned into a wait afterwards.
-            struct Place { uint32_t addr, fbar, ebar, parity; };
-            auto next_ring = [&]() -> Place {
-                Place pl{s_ring + slot * SLOT_BYTES, B.full + 8 * slot, B.empty + 8 * slot, phase};
+            auto wait_full = [&]() -> uint32_t {
+                mbar_wait(B.full + 8 * slot, phase, a.status, &abort_flag, 0x201);
+                const uint32_t s = slot;
                 if (++slot == (uint32_t)lay.nslot) { slot = 0; phase ^= 1u; }
-                return pl;
+                return s;
             };
-            for (int which = which_lo; which < which_hi; ++which) {
+            for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
+                if (which < which_lo || which >= which_hi) continue;
                 const int nj = P.n_jobs[which];
                 for (int j = 0; j < nj; ++j, ++jc) {
                     const TcJob job = P.jobs[which][j];
@@ -490,85 +474,54 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         const uint32_t idesc = make_idesc(256, job.nc);
                         const int aux_lo = job.c0 >> 6, n_pool = lay.nslot + (ks_hid - aux_lo);
                         int r = 0;
-                        // next staging place of this job (same order as the producers)
-                        auto next1 = [&]() -> Place {
-                            Place pl;
+                        // next staging place of this job (same order as the producer): smem address, its empty barrier
+                        auto wait_full1 = [&](uint32_t &addr, uint32_t &ebar) {
                             if (r < lay.nslot) {
-                                pl = next_ring();
+                                const uint32_t sl = wait_full();
+                                addr = s_ring + sl * SLOT_BYTES;
+                                ebar = B.empty + 8 * sl;
                             } else {
                                 const uint32_t x = (uint32_t)(aux_lo + r - lay.nslot);
-                                pl = Place{s_hidden + x * SLOT_BYTES, B.afull + 8 * x, B.aempty + 8 * x, (aux_phase >> x) & 1u};
+                                mbar_wait(B.afull + 8 * x, (aux_phase >> x) & 1u, a.status, &abort_flag, 0x205);
                                 aux_phase ^= 1u << x;
+                                addr = s_hidden + x * SLOT_BYTES;
+                                ebar = B.aempty + 8 * x;
                             }
                             if (++r == n_pool) r = 0;
-                            return pl;
                         };
-                        Place z = next1(), w = next1();
-                        mbar_wait(z.fbar, z.parity, a.status, &abort_flag, 0x201);
-                        mbar_wait(w.fbar, w.parity, a.status, &abort_flag, 0x205);
                         for (int ks = 0; ks < ks1; ++ks) {
-                            Place zn = z, wn = w;
-                            uint32_t okz = 1, okw = 1;
-                            if (ks + 1 < ks1) {
-                                zn = next1();
-                                wn = next1();
-                                okz = mbar_try<false>(zn.fbar, zn.parity);
-                                okw = mbar_try<false>(wn.fbar, wn.parity);
-                            }
+                            uint32_t az, ez, aw, ew2;
+                            wait_full1(az, ez);
+                            wait_full1(aw, ew2);
                             tc_fence_after();
                             if (issuer) {
-                                issue_kslab(acc, make_desc(z.addr), make_desc(w.addr), idesc, min(4, (d - 64 * ks) >> 4),
-                                            ks == 0);
-                                umma_commit_pair(z.ebar);
-                                umma_commit_pair(w.ebar);
+                                issue_kslab(acc, make_desc(az), make_desc(aw), idesc, min(4, (d - 64 * ks) >> 4), ks == 0);
+                                umma_commit_pair(ez);
+                                umma_commit_pair(ew2);
                             }
-                            if (!okz) mbar_wait(zn.fbar, zn.parity, a.status, &abort_flag, 0x201);
-                            if (!okw) mbar_wait(wn.fbar, wn.parity, a.status, &abort_flag, 0x205);
-                            z = zn;
-                            w = wn;
                         }
                     } else {
                         const int ks2 = (m + 63) >> 6;
                         const uint32_t idesc = which == 0 ? make_idesc(256, 64 * job.nh) : make_idesc(256, 256);
                         const bool first_use = job.first != 0;  // first head group of this source
-                        Place w = next_ring();
-                        if (first_use) {
-                            mbar_wait(B.hid_ready, hid_phase & 1u, a.status, &abort_flag, 0x204);
-                            hid_phase ^= 1u;
-                        }
-                        mbar_wait(w.fbar, w.parity, a.status, &abort_flag, 0x201);
                         for (int ks = 0; ks < ks2; ++ks) {
-                            Place wn = w;
-                            uint32_t okw = 1;
-                            if (ks + 1 < ks2) {
-                                wn = next_ring();
-                                okw = mbar_try<false>(wn.fbar, wn.parity);
+                            if (first_use && (ks & 3) == 0) {
+                                const int g = ks >> 2;
+                                mbar_wait(B.hid_ready + 8 * g, (hid_phase >> g) & 1u, a.status, &abort_flag, 0x204);
+                                hid_phase ^= 1u << g;
                             }
+                            const uint32_t sw = wait_full();
                             tc_fence_after();
                             const uint64_t dh = make_desc(s_hidden + ks * SLOT_BYTES);
-                            const uint64_t dw = make_desc(w.addr);
+                            const uint64_t dw = make_desc(s_ring + sw * SLOT_BYTES);
                             const int nk = min(4, (m - 64 * ks) >> 4);
                             if (issuer) {
                                 if (which == 0)
                                     issue_kslab(acc, dh, dw, idesc, nk, ks == 0);
                                 else
                                     issue_kslab(acc, dw, dh, idesc, nk, ks == 0);
-                                umma_commit_pair(w.ebar);
+                                umma_commit_pair(B.empty + 8 * sw);
                             }
-                            if (ks + 1 < ks2) {
-                                if (first_use && ((ks + 1) & 3) == 0) {  // the next slab starts a new hidden chunk
-                                    const int g = (ks + 1) >> 2;
-                                    mbar_wait(B.hid_ready + 8 * g, (hid_phase >> g) & 1u, a.status, &abort_flag, 0x204);
-                                    hid_phase ^= 1u << g;
-                                }
-                                if (!okw) mbar_wait(wn.fbar, wn.parity, a.status, &abort_flag, 0x201);
-                            }
-                            w = wn;
-                        }
-                        // last head group of this source: its hidden slabs may be lent to the ring again
-                        if (j + 1 == nj || P.jobs[which][j + 1].kind == 1) {
-                            if (issuer) umma_commit_pair(B.src_done + 8 * n_done);
-                            ++n_done;
                         }
                     }
                     if (issuer) umma_commit_pair(B.jfull + 8 * buf);
@@ -613,7 +566,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             for (int i = et; i < nq_part * 64; i += 256) qs[i] = __bfloat162float(qg[i]) * a.scale;
         }
         uint32_t jc = 0;
-        for (int which = which_lo; which < which_hi; ++which) {
+        for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
+                if (which < which_lo || which >= which_hi) continue;
             const int nj = P.n_jobs[which];
             if (which == 1 && !lay.kv_split) {
                 // every probability this CTA will read has been written, here and by the peer
@@ -822,9 +776,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     if (kvh >= 0 && tt.valid > 0) {
                         const int ql0 = (kvh - h_lo) * group;
                         const float *Sp = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE;
-                        float2 accv[8], accw[8];
+                        float2 accv[8];
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) accv[g] = accw[g] = make_float2(0.f, 0.f);
+                        for (int g = 0; g < 8; ++g) accv[g] = make_float2(0.f, 0.f);
                         for (int gi = 0; gi < 4; ++gi) {
                             if (32 * gi >= tt.valid) break;
                             float y[32];
@@ -834,19 +788,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 #pragma unroll
                                 for (int t = 0; t < 32; ++t) y[t] = (32 * gi + t < tt.valid) ? y[t] : 0.f;
                             }
-                            // token groups outside, query heads inside: one accumulation chain per head
 #pragma unroll
-                            for (int t = 0; t < 8; ++t) {
-                                const float2 ya = make_float2(y[4 * t], y[4 * t + 1]);
-                                const float2 yb = make_float2(y[4 * t + 2], y[4 * t + 3]);
+                            for (int g = 0; g < 8; ++g) {
+                                if (g < group) {
+                                    const float4 *p4 = reinterpret_cast<const float4 *>(Sp + g * PSTRIDE + 32 * gi);
+                                    float2 s0 = accv[g], s1v = make_float2(0.f, 0.f);
 #pragma unroll
-                                for (int g = 0; g < 8; ++g) {
-                                    if (g < group) {
-                                        const float4 pp =
-                                            *reinterpret_cast<const float4 *>(Sp + g * PSTRIDE + 32 * gi + 4 * t);
-                                        accv[g] = __ffma2_rn(make_float2(pp.x, pp.y), ya, accv[g]);
-                                        accw[g] = __ffma2_rn(make_float2(pp.z, pp.w), yb, accw[g]);
+                                    for (int t = 0; t < 8; ++t) {
+                                        const float4 pp = p4[t];
+                                        s0 = __ffma2_rn(make_float2(pp.x, pp.y), make_float2(y[4 * t], y[4 * t + 1]), s0);
+                                        s1v = __ffma2_rn(make_float2(pp.z, pp.w), make_float2(y[4 * t + 2], y[4 * t + 3]), s1v);
                                     }
+                                    accv[g] = __fadd2_rn(s0, s1v);
                                 }
                             }
                         }
@@ -856,7 +809,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             if (g < group) {
                                 const int qh = (h_lo * group) + ql0 + g;
                                 float *part = a.partials + (((int64_t)tt.si * a.max_chunks + tt.chunk) * hq + qh) * (64 + 2);
-                                part[2 + c] = ((accv[g].x + accv[g].y) + (accw[g].x + accw[g].y)) + bias * Sp[g * PSTRIDE + 128];
+                                part[2 + c] = (accv[g].x + accv[g].y) + bias * Sp[g * PSTRIDE + 128];
                             }
                         }
                     }
