@@ -60,6 +60,7 @@ struct PairLaunch {
     const TcPart *parts;  // this layer's tables for the chosen split: parts[0 .. split-1]
     uint32_t off_hidden, off_ring, off_part, off_fparam, off_q, off_s, off_bar;
     int32_t nslot, max_m, max_in, split, nq_local;
+    int32_t n_pairs;  // tile pairs of this launch; a cluster takes pairs first, first + stride, ...
     // K/V split (small grids): one cluster restores K and publishes the probabilities, another restores V
     int32_t kv_split;
     uint32_t epoch;     // value a probability flag takes in this launch
@@ -229,10 +230,11 @@ struct Bars {
     uint32_t jempty;       // [2] both CTAs' epilogue warps are done reading it (leader)
     uint32_t hid_ready;    // [MAX_HID_GROUPS] hidden columns written by both CTAs (leader)
     uint32_t p_ready;      // [1] both CTAs' probabilities of all K heads are in place (both CTAs)
+    uint32_t s_free;       // [1] the peer's epilogue warps are done reading a pair's probabilities (both CTAs)
     uint32_t afull, aempty;  // [MAX_AUX] hidden slabs lent to the operand ring while they hold no activations
 };
 constexpr int MAX_AUX = 4 * MAX_HID_GROUPS;
-constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 1 + 2 * MAX_AUX;
+constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 2 + 2 * MAX_AUX;
 
 struct TileInfo {
     int si, chunk, valid;  // listed-sequence index, tile index inside the sequence, valid tokens (0 = no tile)
@@ -273,16 +275,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     const uint32_t rank = blockIdx.x & 1u;  // rank in the cluster = which of the pair's two tiles
     const int cid = blockIdx.x >> 1;
     const int per_pair = lay.split * (lay.kv_split ? 2 : 1);  // clusters that share one pair of tiles
-    const int sub = cid % per_pair, pair = cid / per_pair;
+    const int sub = cid % per_pair;
+    const int pair0 = cid / per_pair, pair_stride = (int)(gridDim.x >> 1) / per_pair;
     const int part_i = sub % lay.split;
     // this cluster's share of the work: K only, V only, or K then V
     const int which_lo = lay.kv_split ? sub / lay.split : 0, which_hi = lay.kv_split ? which_lo + 1 : 2;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hq = a.hq, group = a.hq / a.hkv;
     const bool leader = rank == 0;
-
-    const TileInfo tl[2] = {locate_tile(tix, 2 * pair, seqs.n), locate_tile(tix, 2 * pair + 1, seqs.n)};
-    const TileInfo mine = tl[rank];
 
     // carve shared memory (1024-byte aligned for the swizzled tiles; same offsets in both CTAs)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -301,7 +301,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     B.jempty = B.jfull + 16;
     B.hid_ready = B.jempty + 16;
     B.p_ready = B.hid_ready + 8 * MAX_HID_GROUPS;
-    B.afull = B.p_ready + 8;
+    B.s_free = B.p_ready + 8;
+    B.afull = B.s_free + 8;
     B.aempty = B.afull + 8 * MAX_AUX;
 
     {  // this cluster's job tables -> shared memory
@@ -321,6 +322,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         }
         for (int i = 0; i < MAX_HID_GROUPS; ++i) mbar_init(B.hid_ready + 8 * i, 2 * N_EPI_WARPS);
         mbar_init(B.p_ready, 2 * N_EPI_WARPS);
+        mbar_init(B.s_free, N_EPI_WARPS);
         for (int i = 0; i < MAX_AUX; ++i) {
             mbar_init(B.afull + 8 * i, 1);
             mbar_init(B.aempty + 8 * i, 1);
@@ -347,6 +349,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // places and wait for each of them to be free, so both see the same ring state.
         const uint32_t pid = warp == 0 ? 0u : 1u;
         if (lane == 0) {
+            uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0;
+          for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride) {
+            const TileInfo mine = locate_tile(tix, 2 * pair + (int)rank, seqs.n);
             // pool rows of the tile's two 64-token halves (a half with no valid token re-reads a valid row block)
             int row[2] = {0, 0};
             if (mine.valid > 0) {
@@ -358,7 +363,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     row[h] = page * a.page_tokens + t % a.page_tokens;
                 }
             }
-            uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0;
             // wait for the ring slot to be free in this CTA; its owner announces the pair's bytes (leader)
             auto acquire = [&](uint32_t pair_bytes, bool own) -> uint32_t {
                 mbar_wait(B.empty + 8 * slot, phase ^ 1u, a.status, &abort_flag, 0x101);
@@ -444,6 +448,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     }
                 }
             }
+          }  // pairs
         }
     } else if (warp == 1) {
         // ============================== MMA issuer (leader CTA) ==============================
@@ -458,6 +463,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (++slot == (uint32_t)lay.nslot) { slot = 0; phase ^= 1u; }
                 return s;
             };
+          for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride) {
             for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
                 const int nj = P.n_jobs[which];
@@ -528,6 +534,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     __syncwarp();
                 }
             }
+          }  // pairs
         }
     } else if (warp < PRODUCER2_WARP) {
         // ============================== epilogue warps (both CTAs) ==============================
@@ -541,9 +548,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         float *s1 = fparam, *t1 = fparam + m_pad, *b2 = fparam + 2 * m_pad;
         const uint32_t jempty_leader[2] = {map_to_cta(B.jempty, 0), map_to_cta(B.jempty + 8, 0)};
         const uint32_t hid_leader = map_to_cta(B.hid_ready, 0);
+        const int nq_part = (P.h_hi - h_lo) * group;
+        uint32_t jc = 0, it = 0;
+      for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride, ++it) {
+        const TileInfo tl[2] = {locate_tile(tix, 2 * pair, seqs.n), locate_tile(tix, 2 * pair + 1, seqs.n)};
+        const TileInfo mine = tl[rank];
+        bool s_waited = it == 0;  // the peer has finished reading the previous pair's probabilities in its buffer
         const uint32_t peer_S = map_to_cta(smem_u32(Sall), rank ^ 1u);
         float *Smine = Sall + (size_t)rank * lay.nq_local * PSTRIDE;
-        const int nq_part = (P.h_hi - h_lo) * group;
         if (mine.valid > 0) {
             // pull this tile's latent rows of every source from HBM into L2 ahead of the producers' loads
             int item = 0;
@@ -565,7 +577,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)mine.si * hq + h_lo * group) * 64;
             for (int i = et; i < nq_part * 64; i += 256) qs[i] = __bfloat162float(qg[i]) * a.scale;
         }
-        uint32_t jc = 0;
         for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
             const int nj = P.n_jobs[which];
@@ -587,12 +598,26 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 const uint32_t acc = tmem + 256u * buf + tl_addr;
                 if (job.kind == 1) {
                     if (job.first) {
-                        epi_bar_sync();  // everyone is done with the previous source's parameters
-                        for (int i = et; i < m_pad; i += 256) {
-                            s1[i] = i < m ? sp.s1[i] : 0.f;
-                            t1[i] = i < m ? sp.t1[i] : 0.f;
+                        // this source's parameters: fetched into registers first, so that the global-memory
+                        // latency overlaps the wait for the other warps
+                        float ps[MAX_HID_GROUPS], pt[MAX_HID_GROUPS], pb[MAX_HID_GROUPS];
+#pragma unroll
+                        for (int u = 0; u < MAX_HID_GROUPS; ++u) {
+                            const int i = et + 256 * u;
+                            ps[u] = i < m ? sp.s1[i] : 0.f;
+                            pt[u] = i < m ? sp.t1[i] : 0.f;
+                            pb[u] = i < sp.in_dim ? sp.b2[i] : 0.f;
                         }
-                        for (int i = et; i < sp.in_dim; i += 256) b2[i] = sp.b2[i];
+                        epi_bar_sync();  // everyone is done with the previous source's parameters
+#pragma unroll
+                        for (int u = 0; u < MAX_HID_GROUPS; ++u) {
+                            const int i = et + 256 * u;
+                            if (i < m_pad) {
+                                s1[i] = ps[u];
+                                t1[i] = pt[u];
+                            }
+                            if (i < sp.in_dim) b2[i] = pb[u];
+                        }
                         epi_bar_sync();
                     }
                     // ---- bias + BatchNorm + LeakyReLU, bf16, into the swizzled hidden slabs ----
@@ -741,6 +766,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 *reinterpret_cast<float4 *>(grow + 4 * lane) = sc;
                                 if (lane == 0) grow[128] = sum;
                             } else {
+                                if (!s_waited) {
+                                    mbar_wait<false, 100>(B.s_free, (it - 1u) & 1u, a.status, &abort_flag, 0x305);
+                                    s_waited = true;
+                                }
                                 const uint32_t prow = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE) * 4u;
                                 st_cluster_v4(prow + 16u * lane, sc.x, sc.y, sc.z, sc.w);
                                 if (lane == 0) st_cluster_f32(prow + 128u * 4u, sum);
@@ -767,7 +796,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 } else {
                     // V: this thread owns (head place, channel) = row; columns = tokens of tile chalf
                     if (!lay.kv_split && !p_waited) {
-                        mbar_wait<true, 100>(B.p_ready, 0, a.status, &abort_flag, 0x303);
+                        mbar_wait<true, 100>(B.p_ready, it & 1u, a.status, &abort_flag, 0x303);
                         p_waited = true;
                     }
                     const int hp = 2 * (int)rank + (row >> 6), c = row & 63;
@@ -819,6 +848,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 }
             }
         }
+        if (!lay.kv_split) {  // this CTA no longer reads the pair's probabilities: the peer may overwrite them
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(map_to_cta(B.s_free, rank ^ 1u));
+        }
+      }  // pairs
     }
     // ---- teardown: nobody leaves while the peer may still read or write this CTA ----
     tc_fence_before();
@@ -1004,7 +1038,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
             const WhichPlan &wp = plans[l].w[which];
             for (int s = 0; s < wp.n_src && ok; ++s) {
                 const SourcePlan &sp = wp.src[s];
-                if (!sp.compressed || sp.d % 16 || sp.m % 16 || sp.d < 16 || sp.m < 16 || sp.m > 256 * MAX_HID_GROUPS ||
+                if (!sp.compressed || sp.d % 16 || sp.m % 16 || sp.d < 16 || sp.m < 16 || sp.m > 256 * MAX_HID_GROUPS || sp.in_dim > 256 * MAX_HID_GROUPS ||
                     sp.in_dim % 64 || sp.width != sp.d) {
                     ok = false;
                     break;
@@ -1100,6 +1134,7 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     const int nq_local = a.hkv / split * group;
     PairLaunch lay = make_launch(nq_local, lc.max_m, lc.max_in, pick_nslot(nq_local, lc.max_m, lc.max_in));
     lay.split = split;
+    lay.n_pairs = n_pairs;
     lay.kv_split = kv_split;
     lay.epoch = ++tc.epoch;
     lay.pbuf = tc.pbuf;
@@ -1113,7 +1148,10 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
         if (e != cudaSuccess) return e;
         configured_smem = smem;
     }
-    dim3 grid(2 * n_pairs * split * (kv_split ? 2 : 1));
+    // at most one resident cluster per SM pair; clusters walk the pairs with that stride
+    const int per_pair = split * (kv_split ? 2 : 1);
+    const int n_clusters = std::min(n_pairs * per_pair, std::max(per_pair, tc.n_sms / 2 / per_pair * per_pair));
+    dim3 grid(2 * n_clusters);
     decode_pair_kernel<<<grid, NTHREADS, smem, st>>>(a, seqs, tix, lay);
     return cudaGetLastError();
 }
