@@ -30,6 +30,10 @@ if ROOT not in sys.path:
 
 import kvcar_synth as synth  # noqa: E402
 
+# DRAM bytes (read + write) per decode_pair_kernel launch from the ncu capture summarised in
+# profiles/decode_pair_kernel_c2.md (mean of two layers); only for the workload and kernel it was taken on
+NCU_TRAFFIC_BYTES = {("c2_gpt2s_12l_b8_L1024", "auto", False): 27.25e6}
+
 METRIC = "decode tokens/s over latent KV cache"
 UNIT = "tokens/s"
 
@@ -410,6 +414,7 @@ def main():
         ach = flops / (kern_ms / 1e3) / 1e12
         roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None}
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, args.kernel, bool(args.uncompressed)))
     roof.update({"kernel": "decode_attention (decoder + attention + combine)", "launches": n_k,
                  "avg_launch_us": 1e3 * kern_ms / n_k, "peak_source": peaks["source"] + " (sustained)",
                  "algorithmic_flops_per_launch": flops / n_k, "algorithmic_bytes_per_launch": byts / n_k,
