@@ -218,13 +218,16 @@ def oracle_sample(w, src, aes, kept, steps_k, steps_v, steps_q, budget_s, gpu_ou
     t0 = time.perf_counter()
     pairs = 0
     worst = 0.0
-    for q in seqs:
-        for l in range(w.n_layers):
-            o.encode_append(l, [q], 1, steps_k[l][q][None, None], steps_v[l][q][None, None])
-            ref = o.decode_attention(l, [q], steps_q[l][q][None])
-            pairs += 1
-            if gpu_out is not None:
-                worst = max(worst, float(np.max(np.abs(gpu_out[l][q] - ref[0]))))
+    for rep_i in range(8):       # the same step again (appending at an unadvanced position overwrites) until the budget is spent
+        for q in seqs:
+            for l in range(w.n_layers):
+                o.encode_append(l, [q], 1, steps_k[l][q][None, None], steps_v[l][q][None, None])
+                ref = o.decode_attention(l, [q], steps_q[l][q][None])
+                pairs += 1
+                if gpu_out is not None:
+                    worst = max(worst, float(np.max(np.abs(gpu_out[l][q] - ref[0]))))
+            if time.perf_counter() - t0 > budget_s:
+                break
         if time.perf_counter() - t0 > budget_s:
             break
     dt = time.perf_counter() - t0
@@ -339,8 +342,8 @@ def main():
     sess.device = torch.device(f"cuda:{local}")
     seqs = list(range(w.batch))
     do_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
-    keep = tuple(range(min(2, w.batch))) if do_cpu else ()
-    kept = prefill(sess, w, torch, keep)
+    keep = tuple(range(min(8 if w.cached_tokens <= 4096 else 1, w.batch))) if do_cpu else ()
+    prefill(sess, w, torch, ())
     stream = sess.stream()
     flags = B.INCLUDE_CURRENT_EXACT
     total_steps = 2 * (W_ + K_)
@@ -353,12 +356,12 @@ def main():
         torch.cuda.synchronize()
 
     # ---- pass 1: the headline timing --------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()          # nvidia-smi needs a moment to come up: it samples warm-up, timed region and pass 2
     for i in range(W_):
         run_step(sess, w, seqs, k, v, q, out, i, stream, flags)
     sess.ctx.sync_status(stream)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     launches0 = sess.ctx.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_)]
     barrier()
@@ -373,7 +376,6 @@ def main():
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = float(sum(step_ms))
     launches = sess.ctx.launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
     sess.ctx.sync_status(stream)
     if world > 1:
         t = torch.tensor([total_ms], device=sess.device)
@@ -401,6 +403,7 @@ def main():
         sess.ctx.advance(seqs, 1, stream)
     torch.cuda.synchronize()
     sess.ctx.sync_status(stream)
+    clocks = sampler.stop() if rank == 0 else None
     peaks = measured_peaks()
     flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
     byts = sum(sess.ctx.layer_work_per_token(l)[0] * L * w.batch for (l, L, _, _) in kev)
@@ -455,7 +458,7 @@ def main():
 
     # ---- CPU baseline: the oracle on a bounded sample ------------------------
     cpu = None
-    if do_cpu and kept:
+    if do_cpu:
         # a fresh decode step at the prefilled length for the sampled sequences, compared with the GPU
         sess2, _, _ = build_session(w, args, torch, 4)
         kept2 = prefill(sess2, w, torch, keep)
@@ -469,8 +472,9 @@ def main():
         del sess2
         r = oracle_sample(w, src, aes, kept2, sk, sv, sq, args.cpu_seconds, go)
         cpu = {"value": r["value"], "unit": UNIT, "cores": host_threads(), "kind": "oracle",
-               "sample": f"decode step at {w.cached_tokens} cached tokens for {r['pairs']} (sequence, layer) pairs "
-                         f"of {w.batch * w.n_layers} ({r['seconds']:.1f} s), scaled by the pair count",
+               "sample": f"decode step at {w.cached_tokens} cached tokens: {r['pairs']} (sequence, layer) pair evaluations "
+                         f"over {len(keep)} of {w.batch} sequences ({r['seconds']:.1f} s), scaled to the "
+                         f"{w.batch * w.n_layers} pairs of a step",
                "max_abs_err_gpu_vs_oracle_on_sample": r["max_abs_err_vs_gpu"]}
 
     if rank == 0:
