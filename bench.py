@@ -71,6 +71,23 @@ def measured_peaks():
 
 
 # ----------------------------------------------------------------------------
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's figure (replicas run independently; the job is as slow as its slowest replica)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(batch_per_rank: int, steps: int, world: int, seconds: float) -> float:
+    """Replicas only (weak scaling): every rank decodes its own batch; value = all ranks' tokens / slowest time."""
+    return world * batch_per_rank * steps / seconds
+
+
+# ----------------------------------------------------------------------------
 class ClockSampler:
     """nvidia-smi clocks / throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -377,12 +394,9 @@ def main():
     total_ms = float(sum(step_ms))
     launches = sess.ctx.launch_count() - launches0
     sess.ctx.sync_status(stream)
-    if world > 1:
-        t = torch.tensor([total_ms], device=sess.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, sess.device)
     ms_per_step = total_ms / K_
-    value = world * w.batch * K_ / (total_ms / 1e3)
+    value = whole_job_tokens_per_s(w.batch, K_, world, total_ms / 1e3)
 
     # ---- pass 2: the decode kernel alone, per launch ----------------------
     base = W_ + K_
@@ -445,12 +459,9 @@ def main():
             e2e_step()
         barrier()
         e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], device=sess.device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, world, sess.device)
         elem = 2 if w.storage == "bf16" else 4
-        e2e = {"value": world * w.batch * n_e2e / e2e_s, "unit": UNIT, "steps": n_e2e,
+        e2e = {"value": whole_job_tokens_per_s(w.batch, n_e2e, world, e2e_s), "unit": UNIT, "steps": n_e2e,
                "h2d_bytes_per_step": w.n_layers * w.batch * (2 * w.kv_width + w.n_q_heads * w.head_dim) * elem,
                "d2h_bytes_per_step": w.n_layers * w.batch * w.n_q_heads * w.head_dim * elem,
                "timing": "wall clock around K host-buffer steps, stream synchronised every step"}
