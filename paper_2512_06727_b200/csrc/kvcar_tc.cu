@@ -22,9 +22,18 @@
 // written into both CTAs (distributed shared memory) because the V product of a
 // head lands, for both tiles, in the CTA that loaded the head's weight rows.
 //
-// Warp roles: warp 0 = TMA producer (both CTAs), warp 1 = MMA issuer (leader CTA)
-// and tensor-memory owner, warps 2-9 = epilogue (lane quarter = warp % 4, column
-// half = (warp-2) / 4).
+// Grid.  At most one cluster per SM pair; a cluster walks the tile pairs with that
+// stride, so loads and products of the next pair start while the epilogues of the
+// current one finish.  Small grids spread one tile pair over several clusters: K and V
+// on separate clusters (the K cluster publishes each head's probabilities in global
+// memory behind a release/acquire flag), and the layer's KV heads in halves or quarters.
+//
+// Operand staging.  16-KB places: a ring beside the hidden activations, plus, during
+// hidden-chunk jobs, the hidden slabs that hold no activations yet.
+//
+// Warp roles: warps 0 and 10 = TMA producers (both CTAs; they take alternate loads),
+// warp 1 = MMA issuer (leader CTA) and tensor-memory owner, warps 2-9 = epilogue (lane
+// quarter = warp % 4, column half = (warp-2) / 4).
 //
 // All waits are bounded: a wait that runs out records a code in the status word
 // and the kernel carries on to its normal exit (results are then meaningless and

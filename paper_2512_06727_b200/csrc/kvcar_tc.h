@@ -8,7 +8,6 @@ constexpr int TC_MAX_LAYERS = 512;
 constexpr int TC_MAX_SRC = 6;    // distinct source layers per K or V of one head subset
 constexpr int TC_MAX_JOBS = 24;  // accumulator jobs per K or V of one head subset
 constexpr int TC_SPLIT_TILES = 160;  // the K/V split is used only while 2 x tiles <= SM count
-constexpr int TC_MAX_SPLIT = 4;  // a layer's KV heads can be split over up to 4 clusters per tile pair
 
 // One source layer as the tensor-core kernel sees it.
 struct TcSrc {
