@@ -58,6 +58,8 @@ constexpr int N_EPI_WARPS = 8;
 constexpr int PRODUCER2_WARP = 2 + N_EPI_WARPS;  // second TMA producer, after the epilogue warps
 constexpr int NTHREADS = 32 * (PRODUCER2_WARP + 1);
 constexpr int MAX_HID_GROUPS = 4;  // hidden chunks of 256 columns
+constexpr int QBS = 72;    // bf16 per query row in the MMA-operand copy of the queries (padded against bank conflicts)
+constexpr int PBS = 136;   // bf16 per probability row in the MMA-operand copy of the probabilities
 
 struct TileIndex {
     int32_t n_tiles;
@@ -67,7 +69,8 @@ struct TileIndex {
 
 struct PairLaunch {
     const TcPart *parts;  // this layer's tables for the chosen split: parts[0 .. split-1]
-    uint32_t off_hidden, off_ring, off_part, off_fparam, off_q, off_s, off_bar;
+    uint32_t off_hidden, off_ring, off_part, off_fparam, off_q, off_s, off_qb, off_pb, off_bar;
+    int32_t group_mma;  // query groups of more than two heads: attention products on the warp-level tensor op
     int32_t nslot, max_m, max_in, split, nq_local;
     int32_t n_pairs;  // tile pairs of this launch; a cluster takes pairs first, first + stride, ...
     // K/V split (small grids): one cluster restores K and publishes the probabilities, another restores V
@@ -199,6 +202,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
         : "r"(taddr)
         : "memory");
 }
+// 16 lanes x 8*N columns of fp32 in the accumulator-fragment layout of the warp-level MMA: thread t gets, per
+// 8-column block j, rows t/4 (regs 4j, 4j+1) and t/4 + 8 (regs 4j+2, 4j+3), columns 8j + 2*(t%4) + {0, 1}
+__device__ __forceinline__ void tmem_ld_frag_x4(uint32_t taddr, uint32_t *r) {  // 32 columns
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+        "[%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+// D[16 x 8] += A[16 x 16] . B[16 x 8], bf16 operands, fp32 accumulate (warp-level tensor op for the small
+// attention products of a query group)
+__device__ __forceinline__ void mma_16816(float *d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, "
+        "%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // K-major, 128B-swizzled operand tile: rows of 128 B, 8-row groups 1024 B apart
@@ -301,6 +325,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     const TcPart &P = *reinterpret_cast<const TcPart *>(gbase + lay.off_part);
     float *fparam = reinterpret_cast<float *>(gbase + lay.off_fparam);  // s1[max_m], t1[max_m], b2[max_in]
     float *qs = reinterpret_cast<float *>(gbase + lay.off_q);          // [nq_local][64], pre-scaled, own tile's sequence
+    __nv_bfloat16 *qb = reinterpret_cast<__nv_bfloat16 *>(gbase + lay.off_qb);  // same as bf16 [nq_local][QBS]
+    __nv_bfloat16 *Pb = reinterpret_cast<__nv_bfloat16 *>(gbase + lay.off_pb);  // probabilities as bf16 [2][nq_local][PBS]
     float *Sall = reinterpret_cast<float *>(gbase + lay.off_s);        // [2 tiles][nq_local][PSTRIDE]
     const uint32_t s_bar = base + lay.off_bar;
     Bars B;
@@ -564,6 +590,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         const TileInfo mine = tl[rank];
         bool s_waited = it == 0;  // the peer has finished reading the previous pair's probabilities in its buffer
         const uint32_t peer_S = map_to_cta(smem_u32(Sall), rank ^ 1u);
+        const uint32_t peer_Pb = map_to_cta(smem_u32(Pb), rank ^ 1u);
         float *Smine = Sall + (size_t)rank * lay.nq_local * PSTRIDE;
         if (mine.valid > 0) {
             // pull this tile's latent rows of every source from HBM into L2 ahead of the producers' loads
@@ -584,7 +611,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 }
             const __nv_bfloat16 *qg =
                 reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)mine.si * hq + h_lo * group) * 64;
-            for (int i = et; i < nq_part * 64; i += 256) qs[i] = __bfloat162float(qg[i]) * a.scale;
+            for (int i = et; i < nq_part * 64; i += 256) {
+                const float qv = __bfloat162float(qg[i]) * a.scale;
+                qs[i] = qv;
+                if (lay.group_mma) qb[(i >> 6) * QBS + (i & 63)] = __float2bfloat16_rn(qv);
+            }
         }
         for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
@@ -714,6 +745,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         const float4 val = __ldcg(reinterpret_cast<const float4 *>(
                                                       lay.pbuf + ((size_t)tile * hq + h_lo * group + ql) * PSTRIDE) + v4);
                         *reinterpret_cast<float4 *>(Sall + ((size_t)th * lay.nq_local + ql) * PSTRIDE + 4 * v4) = val;
+                        if (lay.group_mma && v4 < 32)
+                            *reinterpret_cast<uint2 *>(Pb + ((size_t)th * lay.nq_local + ql) * PBS + 4 * v4) =
+                                make_uint2(pack_bf16(val.x, val.y), pack_bf16(val.z, val.w));
                     }
                     epi_bar_sync();
                 }
@@ -722,6 +756,62 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (which == 0) {
                     // K: this thread owns token `row` of this CTA's tile; columns = (head place, channel)
                     const int nh = job.nh;
+                    if (lay.group_mma) {
+                        // scores of a query group as a small matrix product on the warp-level tensor op: the restored
+                        // K rows come out of tensor memory already in the A-fragment layout (16 tokens x 16 channels per
+                        // step), the group's queries are the B operand, one 16-token half of the warp's rows at a time
+                        const int n = lane >> 2, kq = 2 * (lane & 3);
+                        for (int hp = chalf; hp < nh; hp += 2) {
+                            const int ql0 = (job.kvh[hp] - h_lo) * group;
+                            const float *bb = b2 + job.slot[hp] * 64 + kq;
+                            uint32_t bq[8];
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                const __nv_bfloat16 *qr = qb + (ql0 + n) * QBS + 16 * ks + kq;
+                                bq[2 * ks] = n < group ? *reinterpret_cast<const uint32_t *>(qr) : 0u;
+                                bq[2 * ks + 1] = n < group ? *reinterpret_cast<const uint32_t *>(qr + 8) : 0u;
+                            }
+                            uint32_t r[2][32];
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const uint32_t ta = acc + ((uint32_t)(16 * h) << 16) + 64u * hp;
+                                tmem_ld_frag_x4(ta, r[h]);
+                                tmem_ld_frag_x4(ta + 32u, r[h] + 16);
+                            }
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float dsc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks) {
+                                    const int j0 = 2 * ks, j1 = 2 * ks + 1;
+                                    const float2 ba = *reinterpret_cast<const float2 *>(bb + 8 * j0);
+                                    const float2 bc = *reinterpret_cast<const float2 *>(bb + 8 * j1);
+                                    const uint32_t a0 = pack_bf16(__uint_as_float(r[h][4 * j0]) + ba.x,
+                                                                  __uint_as_float(r[h][4 * j0 + 1]) + ba.y);
+                                    const uint32_t a1 = pack_bf16(__uint_as_float(r[h][4 * j0 + 2]) + ba.x,
+                                                                  __uint_as_float(r[h][4 * j0 + 3]) + ba.y);
+                                    const uint32_t a2 = pack_bf16(__uint_as_float(r[h][4 * j1]) + bc.x,
+                                                                  __uint_as_float(r[h][4 * j1 + 1]) + bc.y);
+                                    const uint32_t a3 = pack_bf16(__uint_as_float(r[h][4 * j1 + 2]) + bc.x,
+                                                                  __uint_as_float(r[h][4 * j1 + 3]) + bc.y);
+                                    mma_16816(dsc, a0, a1, a2, a3, bq[2 * ks], bq[2 * ks + 1]);
+                                }
+                                // dsc: tokens (n, n + 8) of this half, queries (kq, kq + 1) of the group
+                                const int tok = (int)lane_base + 16 * h + n;
+                                if (kq < group) {
+                                    float *sr = Smine + (ql0 + kq) * PSTRIDE;
+                                    sr[tok] = tok < mine.valid ? dsc[0] : -INFINITY;
+                                    sr[tok + 8] = tok + 8 < mine.valid ? dsc[2] : -INFINITY;
+                                }
+                                if (kq + 1 < group) {
+                                    float *sr = Smine + (ql0 + kq + 1) * PSTRIDE;
+                                    sr[tok] = tok < mine.valid ? dsc[1] : -INFINITY;
+                                    sr[tok + 8] = tok + 8 < mine.valid ? dsc[3] : -INFINITY;
+                                }
+                            }
+                        }
+                    } else
                     for (int hp = chalf; hp < nh; hp += 2) {
                         float y[64];
                         tmem_ld32(acc + 64u * hp, y);
@@ -768,8 +858,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             float sum = (sc.x + sc.y) + (sc.z + sc.w);
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                            *reinterpret_cast<float4 *>(srow + 4 * lane) = sc;
                             const int qh = h_lo * group + ql;
+                            if (lay.group_mma && !lay.kv_split) {
+                                // the V side multiplies on the warp-level tensor op: probabilities as bf16 pairs
+                                if (!s_waited) {
+                                    mbar_wait<false, 100>(B.s_free, (it - 1u) & 1u, a.status, &abort_flag, 0x305);
+                                    s_waited = true;
+                                }
+                                const uint32_t w0 = pack_bf16(sc.x, sc.y), w1 = pack_bf16(sc.z, sc.w);
+                                const uint32_t po = (uint32_t)((rank * lay.nq_local + ql) * PBS + 4 * lane);
+                                *reinterpret_cast<uint2 *>(Pb + po) = make_uint2(w0, w1);
+                                asm volatile("st.shared::cluster.v2.b32 [%0], {%1, %2};" ::"r"(peer_Pb + 2u * po), "r"(w0),
+                                             "r"(w1)
+                                             : "memory");
+                                if (lane == 0)
+                                    st_cluster_f32(peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE + 128) * 4u, sum);
+                            } else {
+                            *reinterpret_cast<float4 *>(srow + 4 * lane) = sc;
                             if (lay.kv_split) {
                                 float *grow = lay.pbuf + ((size_t)(2 * pair + (int)rank) * hq + qh) * PSTRIDE;
                                 *reinterpret_cast<float4 *>(grow + 4 * lane) = sc;
@@ -782,6 +887,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 const uint32_t prow = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE) * 4u;
                                 st_cluster_v4(prow + 16u * lane, sc.x, sc.y, sc.z, sc.w);
                                 if (lane == 0) st_cluster_f32(prow + 128u * 4u, sum);
+                            }
                             }
                             if (lane == 0) {
                                 srow[128] = sum;
@@ -811,6 +917,70 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     const int hp = 2 * (int)rank + (row >> 6), c = row & 63;
                     const int kvh = job.kvh[hp];
                     const TileInfo tt = tl[chalf];
+                    if (lay.group_mma) {
+                        // restored V rows are the A operand straight from tensor memory (16 channels x 16 tokens per
+                        // step), the group's probabilities the B operand; both 16-channel halves of the warp's rows
+                        if (kvh >= 0 && tt.valid > 0) {
+                            const int n = lane >> 2, kq = 2 * (lane & 3);
+                            const int ql0 = (kvh - h_lo) * group;
+                            const __nv_bfloat16 *prow = Pb + ((size_t)chalf * lay.nq_local + ql0 + n) * PBS + kq;
+                            float dv[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                            for (int gi = 0; gi < 4; ++gi) {
+                                if (32 * gi >= tt.valid) break;
+                                uint32_t r[2][16];
+                                tmem_ld_frag_x4(acc + 128u * chalf + 32u * gi, r[0]);
+                                tmem_ld_frag_x4(acc + (16u << 16) + 128u * chalf + 32u * gi, r[1]);
+                                uint32_t bp[4];
+#pragma unroll
+                                for (int ks = 0; ks < 2; ++ks) {
+                                    const __nv_bfloat16 *pr = prow + 32 * gi + 16 * ks;
+                                    bp[2 * ks] = n < group ? *reinterpret_cast<const uint32_t *>(pr) : 0u;
+                                    bp[2 * ks + 1] = n < group ? *reinterpret_cast<const uint32_t *>(pr + 8) : 0u;
+                                }
+                                tmem_ld_wait();
+                                if (32 * gi + 32 > tt.valid) {  // rows past the tile's end may hold anything
+#pragma unroll
+                                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                                        for (int e = 0; e < 16; ++e)
+                                            if (32 * gi + 8 * (e >> 2) + kq + (e & 1) >= tt.valid) r[h][e] = 0u;
+                                }
+#pragma unroll
+                                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                                    for (int ks = 0; ks < 2; ++ks) {
+                                        const int j0 = 2 * ks, j1 = 2 * ks + 1;
+                                        const uint32_t a0 = pack_bf16(__uint_as_float(r[h][4 * j0]),
+                                                                      __uint_as_float(r[h][4 * j0 + 1]));
+                                        const uint32_t a1 = pack_bf16(__uint_as_float(r[h][4 * j0 + 2]),
+                                                                      __uint_as_float(r[h][4 * j0 + 3]));
+                                        const uint32_t a2 = pack_bf16(__uint_as_float(r[h][4 * j1]),
+                                                                      __uint_as_float(r[h][4 * j1 + 1]));
+                                        const uint32_t a3 = pack_bf16(__uint_as_float(r[h][4 * j1 + 2]),
+                                                                      __uint_as_float(r[h][4 * j1 + 3]));
+                                        mma_16816(dv[h], a0, a1, a2, a3, bp[2 * ks], bp[2 * ks + 1]);
+                                    }
+                            }
+                            // dv[h]: channels (n, n + 8) of half h, queries (kq, kq + 1) of the group
+                            const float *Ssum = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE + 128;
+                            const float *bv = b2 + job.slot[hp] * 64;
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                if (kq + e < group) {
+                                    const int qh = h_lo * group + ql0 + kq + e;
+                                    float *part =
+                                        a.partials + (((int64_t)tt.si * a.max_chunks + tt.chunk) * hq + qh) * (64 + 2) + 2;
+                                    const float sum = Ssum[(kq + e) * PSTRIDE];
+#pragma unroll
+                                    for (int h = 0; h < 2; ++h) {
+                                        const int ch = (row & 32) + 16 * h + n;
+                                        part[ch] = dv[h][e] + bv[ch] * sum;
+                                        part[ch + 8] = dv[h][2 + e] + bv[ch + 8] * sum;
+                                    }
+                                }
+                            }
+                        }
+                    } else
                     if (kvh >= 0 && tt.valid > 0) {
                         const int ql0 = (kvh - h_lo) * group;
                         const float *Sp = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE;
@@ -906,7 +1076,7 @@ bool encode_map(EncodeTiledFn fn, void *dst_host, const void *dev_ptr, uint64_t 
 
 inline uint32_t up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-PairLaunch make_launch(int nq_local, int max_m, int max_in, int nslot) {
+PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int nslot) {
     PairLaunch l{};
     const int ks_hid = (max_m + 63) / 64;
     uint32_t o = 0;
@@ -922,6 +1092,11 @@ PairLaunch make_launch(int nq_local, int max_m, int max_in, int nslot) {
     o = up(o + (uint32_t)nq_local * 64 * 4, 16);
     l.off_s = o;
     o = up(o + 2u * (uint32_t)nq_local * PSTRIDE * 4, 16);
+    l.group_mma = group > 2 ? 1 : 0;
+    l.off_qb = o;
+    if (l.group_mma) o = up(o + (uint32_t)nq_local * QBS * 2, 16);
+    l.off_pb = o;
+    if (l.group_mma) o = up(o + 2u * (uint32_t)nq_local * PBS * 2, 16);
     l.off_bar = o;
     l.nslot = nslot;
     l.max_m = max_m;
@@ -932,9 +1107,9 @@ PairLaunch make_launch(int nq_local, int max_m, int max_in, int nslot) {
 uint32_t launch_bytes(const PairLaunch &l) { return l.off_bar + 8u * (2 * l.nslot + N_FIXED_BARS) + 1024u; }
 
 // ring depth that fits beside everything else (0 = does not fit)
-int pick_nslot(int nq_local, int max_m, int max_in) {
+int pick_nslot(int nq_local, int group, int max_m, int max_in) {
     for (int nslot = 10; nslot >= 3; --nslot)
-        if (launch_bytes(make_launch(nq_local, max_m, max_in, nslot)) <= 227u * 1024u) return nslot;
+        if (launch_bytes(make_launch(nq_local, group, max_m, max_in, nslot)) <= 227u * 1024u) return nslot;
     return 0;
 }
 
@@ -1087,7 +1262,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
             const int split = splits[si];
             if (cfg.n_kv_heads % split) continue;
             const int per = cfg.n_kv_heads / split;
-            bool fits = pick_nslot(per * group, max_m, max_in) >= 3;
+            bool fits = pick_nslot(per * group, group, max_m, max_in) >= 3;
             for (int i = 0; i < split && fits; ++i)
                 fits = build_part(plans[l], srcs, i * per, (i + 1) * per, parts[part_index(split, i)]);
             lc.split_ok[si] = fits ? 1 : 0;
@@ -1141,7 +1316,7 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     }
     const int group = a.hq / a.hkv;
     const int nq_local = a.hkv / split * group;
-    PairLaunch lay = make_launch(nq_local, lc.max_m, lc.max_in, pick_nslot(nq_local, lc.max_m, lc.max_in));
+    PairLaunch lay = make_launch(nq_local, group, lc.max_m, lc.max_in, pick_nslot(nq_local, group, lc.max_m, lc.max_in));
     lay.split = split;
     lay.n_pairs = n_pairs;
     lay.kv_split = kv_split;
