@@ -86,15 +86,15 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// arrive on a barrier of any CTA of the cluster (address from map_to_cta), release at cluster scope
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-// same, ordering only this CTA's earlier operations (enough where the data handed over is tensor memory already
-// read, or this CTA's shared memory already fenced for the async proxy)
+// arrive on a barrier of any CTA of the cluster (address from map_to_cta), ordering only this CTA's earlier operations
+// (enough where the data handed over is tensor memory already read, or this CTA's shared memory already fenced for the
+// async proxy)
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
@@ -217,7 +217,7 @@ __device__ __forceinline__ void tmem_ld_frag_x4(uint32_t taddr, uint32_t *r) {  
 // attention products of a query group)
 __device__ __forceinline__ void mma_16816(float *d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                           uint32_t b1) {
-    asm volatile(
+    asm(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, "
         "%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
@@ -240,12 +240,21 @@ __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+// Stores into the peer CTA's shared memory that count their bytes on a barrier there: whoever sees that barrier's
+// phase complete sees the data, with no fence on the writing side.
+__device__ __forceinline__ void st_async_v4(uint32_t addr, uint32_t bar, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+                 "r"(a), "r"(b), "r"(c), "r"(d), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+__device__ __forceinline__ void st_async_v2(uint32_t addr, uint32_t bar, uint32_t a, uint32_t b) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(addr), "r"(a),
+                 "r"(b), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_b32(uint32_t addr, uint32_t bar, uint32_t a) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(addr), "r"(a), "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -286,6 +295,18 @@ __device__ __forceinline__ TileInfo locate_tile(const TileIndex &tix, int tile, 
     const int L = tix.len[lo];
     t.valid = max(0, min(TILE, L - t.chunk * TILE));
     return t;
+}
+
+// head-place fields of a job, picked out of the packed words (no indexed byte arrays in registers)
+__device__ __forceinline__ int job_kvh(const TcJob &j, int hp) {
+    uint32_t w;
+    memcpy(&w, j.kvh, 4);
+    return (int)(int8_t)(w >> (8 * hp));
+}
+__device__ __forceinline__ int job_slot(const TcJob &j, int hp) {
+    uint32_t w;
+    memcpy(&w, j.slot, 4);
+    return (int)(int8_t)(w >> (8 * hp));
 }
 
 // one 64-wide K slab: up to four K=16 steps
@@ -356,7 +377,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             mbar_init(B.jempty + 8 * i, 2 * N_EPI_WARPS);
         }
         for (int i = 0; i < MAX_HID_GROUPS; ++i) mbar_init(B.hid_ready + 8 * i, 2 * N_EPI_WARPS);
-        mbar_init(B.p_ready, 2 * N_EPI_WARPS);
+        mbar_init(B.p_ready, N_EPI_WARPS);
         mbar_init(B.s_free, N_EPI_WARPS);
         for (int i = 0; i < MAX_AUX; ++i) {
             mbar_init(B.afull + 8 * i, 1);
@@ -584,6 +605,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         const uint32_t jempty_leader[2] = {map_to_cta(B.jempty, 0), map_to_cta(B.jempty + 8, 0)};
         const uint32_t hid_leader = map_to_cta(B.hid_ready, 0);
         const int nq_part = (P.h_hi - h_lo) * group;
+        const uint32_t ginv = 65536u / (uint32_t)group + 1u;  // (i * ginv) >> 16 == i / group for the small i used here
         uint32_t jc = 0, it = 0;
       for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride, ++it) {
         const TileInfo tl[2] = {locate_tile(tix, 2 * pair, seqs.n), locate_tile(tix, 2 * pair + 1, seqs.n)};
@@ -591,6 +613,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         bool s_waited = it == 0;  // the peer has finished reading the previous pair's probabilities in its buffer
         const uint32_t peer_S = map_to_cta(smem_u32(Sall), rank ^ 1u);
         const uint32_t peer_Pb = map_to_cta(smem_u32(Pb), rank ^ 1u);
+        const uint32_t peer_pready = map_to_cta(B.p_ready, rank ^ 1u);
         float *Smine = Sall + (size_t)rank * lay.nq_local * PSTRIDE;
         if (mine.valid > 0) {
             // pull this tile's latent rows of every source from HBM into L2 ahead of the producers' loads
@@ -611,22 +634,36 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 }
             const __nv_bfloat16 *qg =
                 reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)mine.si * hq + h_lo * group) * 64;
-            for (int i = et; i < nq_part * 64; i += 256) {
-                const float qv = __bfloat162float(qg[i]) * a.scale;
-                qs[i] = qv;
-                if (lay.group_mma) qb[(i >> 6) * QBS + (i & 63)] = __float2bfloat16_rn(qv);
+            for (int i = 8 * et; i < nq_part * 64; i += 8 * 256) {  // eight elements (16 B) per thread and turn
+                const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(qg + i));
+                const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                float2 f[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    f[u] = __bfloat1622float2(h2[u]);
+                    f[u].x *= a.scale;
+                    f[u].y *= a.scale;
+                }
+                *reinterpret_cast<float4 *>(qs + i) = make_float4(f[0].x, f[0].y, f[1].x, f[1].y);
+                *reinterpret_cast<float4 *>(qs + i + 4) = make_float4(f[2].x, f[2].y, f[3].x, f[3].y);
+                if (lay.group_mma)
+                    *reinterpret_cast<uint4 *>(qb + (i >> 6) * QBS + (i & 63)) =
+                        make_uint4(pack_bf16(f[0].x, f[0].y), pack_bf16(f[1].x, f[1].y), pack_bf16(f[2].x, f[2].y),
+                                   pack_bf16(f[3].x, f[3].y));
             }
         }
         for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
             const int nj = P.n_jobs[which];
             if (which == 1 && !lay.kv_split) {
-                // every probability this CTA will read has been written, here and by the peer
-                asm volatile("fence.acq_rel.cluster;" ::: "memory");
+                // this warp's probabilities are in place here; the peer's arrive as counted bytes, announced by one warp
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_cluster(map_to_cta(B.p_ready, 0));
-                    mbar_arrive_cluster(map_to_cta(B.p_ready, 1));
+                    const uint32_t row_bytes = lay.group_mma ? 128u * 2u + 4u : 128u * 4u + 4u;
+                    if (ew == 0 && tl[rank ^ 1u].valid > 0)
+                        mbar_expect_tx(B.p_ready, (uint32_t)nq_part * row_bytes);
+                    else
+                        mbar_arrive_local(B.p_ready);
                 }
             }
             bool p_waited = false;
@@ -721,7 +758,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     for (int idx = et; idx < n_vec; idx += 256) {
                         const int rrow = idx / (PSTRIDE / 4), v4 = idx % (PSTRIDE / 4);
                         const int th = rrow / rows_per_tile, hp = (rrow % rows_per_tile) / group, g = rrow % group;
-                        const int kvh = job.kvh[hp];
+                        const int kvh = job_kvh(job, hp);
                         if (kvh < 0 || tl[th].valid == 0) continue;
                         const int tile = 2 * pair + th;
                         const uint32_t *fl = lay.pflags + (size_t)tile * a.hkv + kvh;
@@ -762,8 +799,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         // step), the group's queries are the B operand, one 16-token half of the warp's rows at a time
                         const int n = lane >> 2, kq = 2 * (lane & 3);
                         for (int hp = chalf; hp < nh; hp += 2) {
-                            const int ql0 = (job.kvh[hp] - h_lo) * group;
-                            const float *bb = b2 + job.slot[hp] * 64 + kq;
+                            const int ql0 = (job_kvh(job, hp) - h_lo) * group;
+                            const float *bb = b2 + job_slot(job, hp) * 64 + kq;
                             uint32_t bq[8];
 #pragma unroll
                             for (int ks = 0; ks < 4; ++ks) {
@@ -779,14 +816,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 tmem_ld_frag_x4(ta + 32u, r[h] + 16);
                             }
                             tmem_ld_wait();
+                            float dsc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                float dsc[4] = {0.f, 0.f, 0.f, 0.f};
+                            for (int ks = 0; ks < 4; ++ks) {
+                                const int j0 = 2 * ks, j1 = 2 * ks + 1;
+                                const float2 ba = *reinterpret_cast<const float2 *>(bb + 8 * j0);
+                                const float2 bc = *reinterpret_cast<const float2 *>(bb + 8 * j1);
 #pragma unroll
-                                for (int ks = 0; ks < 4; ++ks) {
-                                    const int j0 = 2 * ks, j1 = 2 * ks + 1;
-                                    const float2 ba = *reinterpret_cast<const float2 *>(bb + 8 * j0);
-                                    const float2 bc = *reinterpret_cast<const float2 *>(bb + 8 * j1);
+                                for (int h = 0; h < 2; ++h) {  // two independent accumulator chains
                                     const uint32_t a0 = pack_bf16(__uint_as_float(r[h][4 * j0]) + ba.x,
                                                                   __uint_as_float(r[h][4 * j0 + 1]) + ba.y);
                                     const uint32_t a1 = pack_bf16(__uint_as_float(r[h][4 * j0 + 2]) + ba.x,
@@ -795,8 +832,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                                                   __uint_as_float(r[h][4 * j1 + 1]) + bc.y);
                                     const uint32_t a3 = pack_bf16(__uint_as_float(r[h][4 * j1 + 2]) + bc.x,
                                                                   __uint_as_float(r[h][4 * j1 + 3]) + bc.y);
-                                    mma_16816(dsc, a0, a1, a2, a3, bq[2 * ks], bq[2 * ks + 1]);
+                                    mma_16816(dsc2[h], a0, a1, a2, a3, bq[2 * ks], bq[2 * ks + 1]);
                                 }
+                            }
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const float *dsc = dsc2[h];
                                 // dsc: tokens (n, n + 8) of this half, queries (kq, kq + 1) of the group
                                 const int tok = (int)lane_base + 16 * h + n;
                                 if (kq < group) {
@@ -817,7 +858,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         tmem_ld32(acc + 64u * hp, y);
                         tmem_ld32(acc + 64u * hp + 32u, y + 32);
                         tmem_ld_wait();
-                        const float4 *bb = reinterpret_cast<const float4 *>(b2 + job.slot[hp] * 64);
+                        const float4 *bb = reinterpret_cast<const float4 *>(b2 + job_slot(job, hp) * 64);
                         float2 y2[32];
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
@@ -825,7 +866,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             y2[2 * c] = __fadd2_rn(make_float2(y[4 * c], y[4 * c + 1]), make_float2(b4.x, b4.y));
                             y2[2 * c + 1] = __fadd2_rn(make_float2(y[4 * c + 2], y[4 * c + 3]), make_float2(b4.z, b4.w));
                         }
-                        const int ql0 = (job.kvh[hp] - h_lo) * group;
+                        const int ql0 = (job_kvh(job, hp) - h_lo) * group;
                         for (int g = 0; g < group; ++g) {
                             const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g) * 64);
                             float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
@@ -843,58 +884,77 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     __syncwarp();
                     if (lane == 0) mbar_arrive_remote(jempty_leader[buf]);
                     epi_bar_sync();
-                    // tile softmax of the job's query heads; probabilities go to both CTAs
+                    // tile softmax of the job's query heads, four rows per warp and turn so that their shuffle chains
+                    // overlap; probabilities go to both CTAs
                     if (mine.valid > 0) {
-                        for (int item = ew; item < nh * group; item += N_EPI_WARPS) {
-                            const int hp = item / group;
-                            const int ql = (job.kvh[hp] - h_lo) * group + item % group;
-                            float *srow = Smine + ql * PSTRIDE;
-                            float4 sc = *reinterpret_cast<const float4 *>(srow + 4 * lane);
-                            float mx = fmaxf(fmaxf(sc.x, sc.y), fmaxf(sc.z, sc.w));
+                        const int n_items = nh * group;
+                        for (int base = ew; base < n_items; base += 4 * N_EPI_WARPS) {
+                            int qlv[4];
+                            float4 sc[4];
+                            float mx[4], sum[4];
 #pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                            sc.x = __expf(sc.x - mx); sc.y = __expf(sc.y - mx);
-                            sc.z = __expf(sc.z - mx); sc.w = __expf(sc.w - mx);
-                            float sum = (sc.x + sc.y) + (sc.z + sc.w);
+                            for (int u = 0; u < 4; ++u) {
+                                const int item = base + N_EPI_WARPS * u;
+                                qlv[u] = -1;
+                                sc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (item < n_items) {
+                                    const int hp = (int)(((uint32_t)item * ginv) >> 16);  // item / group
+                                    qlv[u] = (job_kvh(job, hp) - h_lo) * group + (item - hp * group);
+                                    sc[u] = *reinterpret_cast<const float4 *>(Smine + qlv[u] * PSTRIDE + 4 * lane);
+                                }
+                                mx[u] = fmaxf(fmaxf(sc[u].x, sc[u].y), fmaxf(sc[u].z, sc[u].w));
+                            }
 #pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                            const int qh = h_lo * group + ql;
-                            if (lay.group_mma && !lay.kv_split) {
-                                // the V side multiplies on the warp-level tensor op: probabilities as bf16 pairs
-                                if (!s_waited) {
-                                    mbar_wait<false, 100>(B.s_free, (it - 1u) & 1u, a.status, &abort_flag, 0x305);
-                                    s_waited = true;
-                                }
-                                const uint32_t w0 = pack_bf16(sc.x, sc.y), w1 = pack_bf16(sc.z, sc.w);
-                                const uint32_t po = (uint32_t)((rank * lay.nq_local + ql) * PBS + 4 * lane);
-                                *reinterpret_cast<uint2 *>(Pb + po) = make_uint2(w0, w1);
-                                asm volatile("st.shared::cluster.v2.b32 [%0], {%1, %2};" ::"r"(peer_Pb + 2u * po), "r"(w0),
-                                             "r"(w1)
-                                             : "memory");
-                                if (lane == 0)
-                                    st_cluster_f32(peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE + 128) * 4u, sum);
-                            } else {
-                            *reinterpret_cast<float4 *>(srow + 4 * lane) = sc;
-                            if (lay.kv_split) {
-                                float *grow = lay.pbuf + ((size_t)(2 * pair + (int)rank) * hq + qh) * PSTRIDE;
-                                *reinterpret_cast<float4 *>(grow + 4 * lane) = sc;
-                                if (lane == 0) grow[128] = sum;
-                            } else {
-                                if (!s_waited) {
-                                    mbar_wait<false, 100>(B.s_free, (it - 1u) & 1u, a.status, &abort_flag, 0x305);
-                                    s_waited = true;
-                                }
-                                const uint32_t prow = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE) * 4u;
-                                st_cluster_v4(prow + 16u * lane, sc.x, sc.y, sc.z, sc.w);
-                                if (lane == 0) st_cluster_f32(prow + 128u * 4u, sum);
+                            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __shfl_xor_sync(0xffffffffu, mx[u], o));
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                sc[u].x = __expf(sc[u].x - mx[u]); sc[u].y = __expf(sc[u].y - mx[u]);
+                                sc[u].z = __expf(sc[u].z - mx[u]); sc[u].w = __expf(sc[u].w - mx[u]);
+                                sum[u] = (sc[u].x + sc[u].y) + (sc[u].z + sc[u].w);
                             }
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], o);
+                            if (!lay.kv_split && !s_waited) {
+                                // the peer has read the previous pair's probabilities out of its copy
+                                mbar_wait<false, 100>(B.s_free, (it - 1u) & 1u, a.status, &abort_flag, 0x305);
+                                s_waited = true;
                             }
-                            if (lane == 0) {
-                                srow[128] = sum;
-                                float *part =
-                                    a.partials + (((int64_t)mine.si * a.max_chunks + mine.chunk) * hq + qh) * (64 + 2);
-                                part[0] = mx;
-                                part[1] = sum;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int ql = qlv[u];
+                                if (ql < 0) continue;
+                                const int qh = h_lo * group + ql;
+                                float *srow = Smine + ql * PSTRIDE;
+                                // the peer's copy is written with stores that count their bytes on the peer's barrier
+                                const uint32_t psum = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE + 128) * 4u;
+                                if (lay.kv_split) {
+                                    float *grow = lay.pbuf + ((size_t)(2 * pair + (int)rank) * hq + qh) * PSTRIDE;
+                                    *reinterpret_cast<float4 *>(grow + 4 * lane) = sc[u];
+                                    if (lane == 0) grow[128] = sum[u];
+                                } else if (lay.group_mma) {
+                                    // the V side multiplies on the warp-level tensor op: probabilities as bf16 pairs
+                                    const uint32_t w0 = pack_bf16(sc[u].x, sc[u].y), w1 = pack_bf16(sc[u].z, sc[u].w);
+                                    const uint32_t po = (uint32_t)((rank * lay.nq_local + ql) * PBS + 4 * lane);
+                                    *reinterpret_cast<uint2 *>(Pb + po) = make_uint2(w0, w1);
+                                    st_async_v2(peer_Pb + 2u * po, peer_pready, w0, w1);
+                                    if (lane == 0) st_async_b32(psum, peer_pready, __float_as_uint(sum[u]));
+                                } else {
+                                    *reinterpret_cast<float4 *>(srow + 4 * lane) = sc[u];
+                                    st_async_v4(psum - 128u * 4u + 16u * lane, peer_pready, __float_as_uint(sc[u].x),
+                                                __float_as_uint(sc[u].y), __float_as_uint(sc[u].z), __float_as_uint(sc[u].w));
+                                    if (lane == 0) st_async_b32(psum, peer_pready, __float_as_uint(sum[u]));
+                                }
+                                if (lane == 0) {
+                                    srow[128] = sum[u];
+                                    float *part =
+                                        a.partials + (((int64_t)mine.si * a.max_chunks + mine.chunk) * hq + qh) * (64 + 2);
+                                    part[0] = mx[u];
+                                    part[1] = sum[u];
+                                }
                             }
                         }
                     }
@@ -904,18 +964,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         epi_bar_sync();
                         if (et < nh && mine.valid > 0)
                             asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(lay.pflags + (size_t)(2 * pair + (int)rank) *
-                                                                                        a.hkv + job.kvh[et]),
+                                                                                        a.hkv + job_kvh(job, et)),
                                          "r"(lay.epoch)
                                          : "memory");
                     }
                 } else {
                     // V: this thread owns (head place, channel) = row; columns = tokens of tile chalf
                     if (!lay.kv_split && !p_waited) {
-                        mbar_wait<true, 100>(B.p_ready, it & 1u, a.status, &abort_flag, 0x303);
+                        mbar_wait<false, 100>(B.p_ready, it & 1u, a.status, &abort_flag, 0x303);
                         p_waited = true;
                     }
                     const int hp = 2 * (int)rank + (row >> 6), c = row & 63;
-                    const int kvh = job.kvh[hp];
+                    const int kvh = job_kvh(job, hp);
                     const TileInfo tt = tl[chalf];
                     if (lay.group_mma) {
                         // restored V rows are the A operand straight from tensor memory (16 channels x 16 tokens per
@@ -946,9 +1006,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                             if (32 * gi + 8 * (e >> 2) + kq + (e & 1) >= tt.valid) r[h][e] = 0u;
                                 }
 #pragma unroll
-                                for (int h = 0; h < 2; ++h)
+                                for (int ks = 0; ks < 2; ++ks)
 #pragma unroll
-                                    for (int ks = 0; ks < 2; ++ks) {
+                                    for (int h = 0; h < 2; ++h) {
                                         const int j0 = 2 * ks, j1 = 2 * ks + 1;
                                         const uint32_t a0 = pack_bf16(__uint_as_float(r[h][4 * j0]),
                                                                       __uint_as_float(r[h][4 * j0 + 1]));
@@ -963,7 +1023,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             }
                             // dv[h]: channels (n, n + 8) of half h, queries (kq, kq + 1) of the group
                             const float *Ssum = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE + 128;
-                            const float *bv = b2 + job.slot[hp] * 64;
+                            const float *bv = b2 + job_slot(job, hp) * 64;
 #pragma unroll
                             for (int e = 0; e < 2; ++e) {
                                 if (kq + e < group) {
@@ -1011,7 +1071,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 }
                             }
                         }
-                        const float bias = b2[job.slot[hp] * 64 + c];
+                        const float bias = b2[job_slot(job, hp) * 64 + c];
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
                             if (g < group) {
