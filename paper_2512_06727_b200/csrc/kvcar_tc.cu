@@ -92,6 +92,10 @@ __device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// arrive on a barrier of any CTA of the cluster (address from map_to_cta), release at cluster scope
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
 // arrive on a barrier of any CTA of the cluster (address from map_to_cta), ordering only this CTA's earlier operations
 // (enough where the data handed over is tensor memory already read, or this CTA's shared memory already fenced for the
 // async proxy)
@@ -240,21 +244,21 @@ __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Stores into the peer CTA's shared memory that count their bytes on a barrier there: whoever sees that barrier's
-// phase complete sees the data, with no fence on the writing side.
-__device__ __forceinline__ void st_async_v4(uint32_t addr, uint32_t bar, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
-                 "r"(a), "r"(b), "r"(c), "r"(d), "r"(bar)
+// Copy `bytes` (a multiple of 16, both addresses 16-byte aligned) from this CTA's shared memory into the peer CTA's
+// and count them on a barrier there: whoever sees that barrier's phase complete sees the data, with no fence on
+// the writing side beyond the one that shows the source to the copy engine.
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     dst_cluster),
+                 "r"(src_cta), "r"(bytes), "r"(bar_cluster)
                  : "memory");
 }
-__device__ __forceinline__ void st_async_v2(uint32_t addr, uint32_t bar, uint32_t a, uint32_t b) {
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(addr), "r"(a),
-                 "r"(b), "r"(bar)
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
                  : "memory");
 }
-__device__ __forceinline__ void st_async_b32(uint32_t addr, uint32_t bar, uint32_t a) {
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(addr), "r"(a), "r"(bar)
-                 : "memory");
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -270,13 +274,13 @@ struct Bars {
     uint32_t full, empty;  // [nslot] each (8 B apart); `full` is used in the leader CTA only
     uint32_t jfull;        // [2] accumulator buffer holds a finished job (both CTAs)
     uint32_t jempty;       // [2] both CTAs' epilogue warps are done reading it (leader)
-    uint32_t hid_ready;    // [MAX_HID_GROUPS] hidden columns written by both CTAs (leader)
+    uint32_t hid_ready;    // [MAX_AUX] one per 64-column hidden slab: written by both CTAs (leader)
     uint32_t p_ready;      // [1] both CTAs' probabilities of all K heads are in place (both CTAs)
     uint32_t s_free;       // [1] the peer's epilogue warps are done reading a pair's probabilities (both CTAs)
     uint32_t afull, aempty;  // [MAX_AUX] hidden slabs lent to the operand ring while they hold no activations
 };
 constexpr int MAX_AUX = 4 * MAX_HID_GROUPS;
-constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_HID_GROUPS + 2 + 2 * MAX_AUX;
+constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_AUX + 2 + 2 * MAX_AUX;
 
 struct TileInfo {
     int si, chunk, valid;  // listed-sequence index, tile index inside the sequence, valid tokens (0 = no tile)
@@ -319,6 +323,11 @@ __device__ __forceinline__ void issue_kslab(uint32_t d_tmem, uint64_t a_desc, ui
 }
 
 // ---------------------------------------------------------------------------- the kernel
+// GMMA: query groups of more than two heads, whose attention products run on the warp-level tensor op (a separate
+// instantiation, so that the code of the other shapes carries none of it)
+// SLAB: no hidden layer of the launch is wider than one chunk; its activations are then handed to the second layer's
+// products slab by slab (the polls this costs the issuing thread are compiled out otherwise)
+template <bool GMMA, bool SLAB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     decode_pair_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ SeqList seqs,
                        const __grid_constant__ TileIndex tix, const __grid_constant__ PairLaunch lay) {
@@ -356,7 +365,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     B.jfull = B.empty + 8 * lay.nslot;
     B.jempty = B.jfull + 16;
     B.hid_ready = B.jempty + 16;
-    B.p_ready = B.hid_ready + 8 * MAX_HID_GROUPS;
+    B.p_ready = B.hid_ready + 8 * MAX_AUX;
     B.s_free = B.p_ready + 8;
     B.afull = B.s_free + 8;
     B.aempty = B.afull + 8 * MAX_AUX;
@@ -376,8 +385,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             mbar_init(B.jfull + 8 * i, 1);
             mbar_init(B.jempty + 8 * i, 2 * N_EPI_WARPS);
         }
-        for (int i = 0; i < MAX_HID_GROUPS; ++i) mbar_init(B.hid_ready + 8 * i, 2 * N_EPI_WARPS);
-        mbar_init(B.p_ready, N_EPI_WARPS);
+        for (int i = 0; i < MAX_AUX; ++i) mbar_init(B.hid_ready + 8 * i, 2 * N_EPI_WARPS);
+        mbar_init(B.p_ready, GMMA ? N_EPI_WARPS : 2 * N_EPI_WARPS);
         mbar_init(B.s_free, N_EPI_WARPS);
         for (int i = 0; i < MAX_AUX; ++i) {
             mbar_init(B.afull + 8 * i, 1);
@@ -566,11 +575,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         const int ks2 = (m + 63) >> 6;
                         const uint32_t idesc = which == 0 ? make_idesc(256, 64 * job.nh) : make_idesc(256, 256);
                         const bool first_use = job.first != 0;  // first head group of this source
+                        constexpr bool slabwise = SLAB;
                         for (int ks = 0; ks < ks2; ++ks) {
-                            if (first_use && (ks & 3) == 0) {
-                                const int g = ks >> 2;
-                                mbar_wait(B.hid_ready + 8 * g, (hid_phase >> g) & 1u, a.status, &abort_flag, 0x204);
-                                hid_phase ^= 1u << g;
+                            if (first_use) {
+                                // Hidden layers of one chunk are announced slab by slab (nothing else hides their
+                                // epilogue); each poll costs tensor time, so wider ones are waited for chunk by chunk,
+                                // through the chunk's last slab.
+                                if (slabwise || (ks & 3) == 0) {
+                                    const int ws = slabwise ? ks : min(ks + 3, ks2 - 1);
+                                    mbar_wait(B.hid_ready + 8 * ws, (hid_phase >> ws) & 1u, a.status, &abort_flag, 0x204);
+                                    hid_phase ^= 1u << ws;
+                                }
                             }
                             const uint32_t sw = wait_full();
                             tc_fence_after();
@@ -646,7 +661,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 }
                 *reinterpret_cast<float4 *>(qs + i) = make_float4(f[0].x, f[0].y, f[1].x, f[1].y);
                 *reinterpret_cast<float4 *>(qs + i + 4) = make_float4(f[2].x, f[2].y, f[3].x, f[3].y);
-                if (lay.group_mma)
+                if (GMMA)
                     *reinterpret_cast<uint4 *>(qb + (i >> 6) * QBS + (i & 63)) =
                         make_uint4(pack_bf16(f[0].x, f[0].y), pack_bf16(f[1].x, f[1].y), pack_bf16(f[2].x, f[2].y),
                                    pack_bf16(f[3].x, f[3].y));
@@ -656,14 +671,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (which < which_lo || which >= which_hi) continue;
             const int nj = P.n_jobs[which];
             if (which == 1 && !lay.kv_split) {
-                // this warp's probabilities are in place here; the peer's arrive as counted bytes, announced by one warp
-                __syncwarp();
-                if (lane == 0) {
-                    const uint32_t row_bytes = lay.group_mma ? 128u * 2u + 4u : 128u * 4u + 4u;
-                    if (ew == 0 && tl[rank ^ 1u].valid > 0)
-                        mbar_expect_tx(B.p_ready, (uint32_t)nq_part * row_bytes);
-                    else
-                        mbar_arrive_local(B.p_ready);
+                if (GMMA) {
+                    // this warp's probabilities are in place here; the peer's arrive as counted bytes, announced by one warp
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (ew == 0 && tl[rank ^ 1u].valid > 0)
+                            mbar_expect_tx(B.p_ready, (uint32_t)nq_part * PBS * 2u);  // whole rows, see the softmax
+                        else
+                            mbar_arrive_local(B.p_ready);
+                    }
+                } else {
+                    // every probability this CTA will read has been written, here and by the peer
+                    asm volatile("fence.acq_rel.cluster;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive_cluster(map_to_cta(B.p_ready, 0));
+                        mbar_arrive_cluster(map_to_cta(B.p_ready, 1));
+                    }
                 }
             }
             bool p_waited = false;
@@ -702,8 +726,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     const bool lr_max = sp.slope <= 1.f;
                     mbar_wait<false, 100>(B.jfull + 8 * buf, (jc >> 1) & 1u, a.status, &abort_flag, 0x301);
                     tc_fence_after();
-                    const int ngroups = (job.nc + 31) >> 5;
-                    for (int g = chalf; g < ngroups; g += 2) {
+                    // One 64-column slab at a time, this warp its half of it.  A hidden layer of a single chunk announces
+                    // each slab as soon as it is written, so that the second layer's products start under the rest of
+                    // this epilogue; a wider one announces each chunk once, through its last slab.
+                    const int ngroups = (job.nc + 31) >> 5, nslabs = (job.nc + 63) >> 6;
+                    constexpr bool slabwise = SLAB;
+                    for (int sl = 0; sl < nslabs; ++sl) {
+                        const int g = 2 * sl + chalf;
+                        if (g < ngroups) {
                         float v[32];
                         tmem_ld32(acc + 32u * g, v);
                         tmem_ld_wait();
@@ -740,13 +770,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                              : "memory");
                             }
                         }
+                        }
+                        if (slabwise) {
+                            fence_async_smem();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_remote(hid_leader + 8u * (uint32_t)((job.c0 >> 6) + sl));
+                        }
                     }
                     tc_fence_before();
-                    fence_async_smem();
+                    if (!slabwise) fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
                         mbar_arrive_remote(jempty_leader[buf]);
-                        mbar_arrive_remote(hid_leader + 8u * (uint32_t)(job.c0 >> 8));
+                        if (!slabwise) mbar_arrive_remote(hid_leader + 8u * (uint32_t)((job.c0 >> 6) + nslabs - 1));
                     }
                     continue;
                 }
@@ -782,9 +818,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         const float4 val = __ldcg(reinterpret_cast<const float4 *>(
                                                       lay.pbuf + ((size_t)tile * hq + h_lo * group + ql) * PSTRIDE) + v4);
                         *reinterpret_cast<float4 *>(Sall + ((size_t)th * lay.nq_local + ql) * PSTRIDE + 4 * v4) = val;
-                        if (lay.group_mma && v4 < 32)
-                            *reinterpret_cast<uint2 *>(Pb + ((size_t)th * lay.nq_local + ql) * PBS + 4 * v4) =
-                                make_uint2(pack_bf16(val.x, val.y), pack_bf16(val.z, val.w));
+                        if (GMMA) {
+                            __nv_bfloat16 *prow = Pb + ((size_t)th * lay.nq_local + ql) * PBS;
+                            if (v4 < 32)
+                                *reinterpret_cast<uint2 *>(prow + 4 * v4) =
+                                    make_uint2(pack_bf16(val.x, val.y), pack_bf16(val.z, val.w));
+                            else
+                                *reinterpret_cast<float *>(prow + 128) = val.x;  // the row's sum
+                        }
                     }
                     epi_bar_sync();
                 }
@@ -793,7 +834,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (which == 0) {
                     // K: this thread owns token `row` of this CTA's tile; columns = (head place, channel)
                     const int nh = job.nh;
-                    if (lay.group_mma) {
+                    if (GMMA) {
                         // scores of a query group as a small matrix product on the warp-level tensor op: the restored
                         // K rows come out of tensor memory already in the A-fragment layout (16 tokens x 16 channels per
                         // step), the group's queries are the B operand, one 16-token half of the warp's rows at a time
@@ -884,16 +925,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     __syncwarp();
                     if (lane == 0) mbar_arrive_remote(jempty_leader[buf]);
                     epi_bar_sync();
-                    // tile softmax of the job's query heads, four rows per warp and turn so that their shuffle chains
-                    // overlap; probabilities go to both CTAs
+                    // tile softmax of the job's query heads; probabilities go to both CTAs.  A query group has several
+                    // rows per warp: four per turn, so that their shuffle chains overlap
                     if (mine.valid > 0) {
+                        constexpr int R = GMMA ? 4 : 1;
                         const int n_items = nh * group;
-                        for (int base = ew; base < n_items; base += 4 * N_EPI_WARPS) {
-                            int qlv[4];
-                            float4 sc[4];
-                            float mx[4], sum[4];
+                        for (int base = ew; base < n_items; base += R * N_EPI_WARPS) {
+                            int qlv[R];
+                            float4 sc[R];
+                            float mx[R], sum[R];
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < R; ++u) {
                                 const int item = base + N_EPI_WARPS * u;
                                 qlv[u] = -1;
                                 sc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -907,9 +949,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __shfl_xor_sync(0xffffffffu, mx[u], o));
+                                for (int u = 0; u < R; ++u) mx[u] = fmaxf(mx[u], __shfl_xor_sync(0xffffffffu, mx[u], o));
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < R; ++u) {
                                 sc[u].x = __expf(sc[u].x - mx[u]); sc[u].y = __expf(sc[u].y - mx[u]);
                                 sc[u].z = __expf(sc[u].z - mx[u]); sc[u].w = __expf(sc[u].w - mx[u]);
                                 sum[u] = (sc[u].x + sc[u].y) + (sc[u].z + sc[u].w);
@@ -917,43 +959,53 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], o);
+                                for (int u = 0; u < R; ++u) sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], o);
                             if (!lay.kv_split && !s_waited) {
                                 // the peer has read the previous pair's probabilities out of its copy
                                 mbar_wait<false, 100>(B.s_free, (it - 1u) & 1u, a.status, &abort_flag, 0x305);
                                 s_waited = true;
                             }
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < R; ++u) {
                                 const int ql = qlv[u];
                                 if (ql < 0) continue;
                                 const int qh = h_lo * group + ql;
                                 float *srow = Smine + ql * PSTRIDE;
-                                // the peer's copy is written with stores that count their bytes on the peer's barrier
-                                const uint32_t psum = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE + 128) * 4u;
                                 if (lay.kv_split) {
                                     float *grow = lay.pbuf + ((size_t)(2 * pair + (int)rank) * hq + qh) * PSTRIDE;
                                     *reinterpret_cast<float4 *>(grow + 4 * lane) = sc[u];
                                     if (lane == 0) grow[128] = sum[u];
-                                } else if (lay.group_mma) {
-                                    // the V side multiplies on the warp-level tensor op: probabilities as bf16 pairs
-                                    const uint32_t w0 = pack_bf16(sc[u].x, sc[u].y), w1 = pack_bf16(sc[u].z, sc[u].w);
-                                    const uint32_t po = (uint32_t)((rank * lay.nq_local + ql) * PBS + 4 * lane);
-                                    *reinterpret_cast<uint2 *>(Pb + po) = make_uint2(w0, w1);
-                                    st_async_v2(peer_Pb + 2u * po, peer_pready, w0, w1);
-                                    if (lane == 0) st_async_b32(psum, peer_pready, __float_as_uint(sum[u]));
+                                } else if (GMMA) {
+                                    // the V side multiplies on the warp-level tensor op: probabilities as bf16 pairs, the
+                                    // row's sum in the row's padding
+                                    __nv_bfloat16 *prow = Pb + (rank * lay.nq_local + ql) * PBS;
+                                    *reinterpret_cast<uint2 *>(prow + 4 * lane) =
+                                        make_uint2(pack_bf16(sc[u].x, sc[u].y), pack_bf16(sc[u].z, sc[u].w));
+                                    if (lane == 0) *reinterpret_cast<float *>(prow + 128) = sum[u];
                                 } else {
                                     *reinterpret_cast<float4 *>(srow + 4 * lane) = sc[u];
-                                    st_async_v4(psum - 128u * 4u + 16u * lane, peer_pready, __float_as_uint(sc[u].x),
-                                                __float_as_uint(sc[u].y), __float_as_uint(sc[u].z), __float_as_uint(sc[u].w));
-                                    if (lane == 0) st_async_b32(psum, peer_pready, __float_as_uint(sum[u]));
+                                    if (lane == 0) srow[128] = sum[u];
+                                    const uint32_t prow = peer_S + (uint32_t)((rank * lay.nq_local + ql) * PSTRIDE) * 4u;
+                                    st_cluster_v4(prow + 16u * lane, sc[u].x, sc[u].y, sc[u].z, sc[u].w);
+                                    if (lane == 0) st_cluster_f32(prow + 128u * 4u, sum[u]);
                                 }
                                 if (lane == 0) {
-                                    srow[128] = sum[u];
                                     float *part =
                                         a.partials + (((int64_t)mine.si * a.max_chunks + mine.chunk) * hq + qh) * (64 + 2);
                                     part[0] = mx[u];
                                     part[1] = sum[u];
+                                }
+                            }
+                            if (GMMA && !lay.kv_split) {
+                                // the finished rows go to the peer whole (probabilities and sum), one copy per row
+                                fence_async_smem();
+                                __syncwarp();
+                                int ql = -1;
+#pragma unroll
+                                for (int u = 0; u < R; ++u) ql = lane == u ? qlv[u] : ql;
+                                if (ql >= 0) {
+                                    const uint32_t off = (uint32_t)((rank * lay.nq_local + ql) * PBS) * 2u;
+                                    bulk_copy_to_peer(peer_Pb + off, smem_u32(Pb) + off, PBS * 2u, peer_pready);
                                 }
                             }
                         }
@@ -971,13 +1023,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 } else {
                     // V: this thread owns (head place, channel) = row; columns = tokens of tile chalf
                     if (!lay.kv_split && !p_waited) {
-                        mbar_wait<false, 100>(B.p_ready, it & 1u, a.status, &abort_flag, 0x303);
+                        mbar_wait<!GMMA, 100>(B.p_ready, it & 1u, a.status, &abort_flag, 0x303);
                         p_waited = true;
                     }
                     const int hp = 2 * (int)rank + (row >> 6), c = row & 63;
                     const int kvh = job_kvh(job, hp);
                     const TileInfo tt = tl[chalf];
-                    if (lay.group_mma) {
+                    if (GMMA) {
                         // restored V rows are the A operand straight from tensor memory (16 channels x 16 tokens per
                         // step), the group's probabilities the B operand; both 16-channel halves of the warp's rows
                         if (kvh >= 0 && tt.valid > 0) {
@@ -1022,7 +1074,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                     }
                             }
                             // dv[h]: channels (n, n + 8) of half h, queries (kq, kq + 1) of the group
-                            const float *Ssum = Sall + ((size_t)chalf * lay.nq_local + ql0) * PSTRIDE + 128;
+                            const __nv_bfloat16 *psum = Pb + ((size_t)chalf * lay.nq_local + ql0) * PBS + 128;
                             const float *bv = b2 + job_slot(job, hp) * 64;
 #pragma unroll
                             for (int e = 0; e < 2; ++e) {
@@ -1030,7 +1082,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                     const int qh = h_lo * group + ql0 + kq + e;
                                     float *part =
                                         a.partials + (((int64_t)tt.si * a.max_chunks + tt.chunk) * hq + qh) * (64 + 2) + 2;
-                                    const float sum = Ssum[(kq + e) * PSTRIDE];
+                                    const float sum = *reinterpret_cast<const float *>(psum + (kq + e) * PBS);
 #pragma unroll
                                     for (int h = 0; h < 2; ++h) {
                                         const int ch = (row & 32) + 16 * h + n;
@@ -1386,17 +1438,21 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * 7 + part_index(split, 0);
     // never less than half an SM's shared memory: two CTAs on one SM would both want all of tensor memory
     const int smem = (int)std::max(launch_bytes(lay), 120u * 1024u);
-    static int configured_smem = 0;
-    if (smem > configured_smem) {
-        cudaError_t e = cudaFuncSetAttribute(decode_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        configured_smem = smem;
-    }
     // at most one resident cluster per SM pair; clusters walk the pairs with that stride
     const int per_pair = split * (kv_split ? 2 : 1);
     const int n_clusters = std::min(n_pairs * per_pair, std::max(per_pair, tc.n_sms / 2 / per_pair * per_pair));
     dim3 grid(2 * n_clusters);
-    decode_pair_kernel<<<grid, NTHREADS, smem, st>>>(a, seqs, tix, lay);
+    using Kernel = void (*)(const DecodeArgs, const SeqList, const TileIndex, const PairLaunch);
+    static const Kernel kernels[4] = {decode_pair_kernel<false, false>, decode_pair_kernel<false, true>,
+                                      decode_pair_kernel<true, false>, decode_pair_kernel<true, true>};
+    static int configured_smem[4] = {0, 0, 0, 0};
+    const int ki = (lay.group_mma ? 2 : 0) + (lc.max_m <= 256 ? 1 : 0);
+    if (smem > configured_smem[ki]) {
+        cudaError_t e = cudaFuncSetAttribute(kernels[ki], cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured_smem[ki] = smem;
+    }
+    kernels[ki]<<<grid, NTHREADS, smem, st>>>(a, seqs, tix, lay);
     return cudaGetLastError();
 }
 
