@@ -616,22 +616,33 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         const int row = lane_base + lane;             // accumulator row of this thread
         const uint32_t tl_addr = lane_base << 16;
         const int m_pad = (lay.max_m + 31) & ~31;  // scale/shift rows are read in whole 32-column groups
-        float *s1 = fparam, *t1 = fparam + m_pad, *b2 = fparam + 2 * m_pad;
+        float *s1 = fparam, *t1 = fparam + m_pad, *b2 = fparam + 2 * m_pad;  // SLAB builds: re-pointed per source
         const uint32_t jempty_leader[2] = {map_to_cta(B.jempty, 0), map_to_cta(B.jempty + 8, 0)};
         const uint32_t hid_leader = map_to_cta(B.hid_ready, 0);
         const int nq_part = (P.h_hi - h_lo) * group;
         const uint32_t ginv = 65536u / (uint32_t)group + 1u;  // (i * ginv) >> 16 == i / group for the small i used here
         uint32_t jc = 0, it = 0;
+        TileInfo tl_next[2] = {};
+        bool next_ready = false;  // tl_next and the queries in shared memory belong to the coming pair
       for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride, ++it) {
-        const TileInfo tl[2] = {locate_tile(tix, 2 * pair, seqs.n), locate_tile(tix, 2 * pair + 1, seqs.n)};
+        // With small autoencoders the start of a pair (finding the tiles, fetching the queries) is a visible share of
+        // the pair's time: there it is done for the next pair while this pair's last products run (SLAB builds).
+        TileInfo tl[2];
+        if (SLAB && next_ready) {
+            tl[0] = tl_next[0];
+            tl[1] = tl_next[1];
+        } else {
+            tl[0] = locate_tile(tix, 2 * pair, seqs.n);
+            tl[1] = locate_tile(tix, 2 * pair + 1, seqs.n);
+        }
         const TileInfo mine = tl[rank];
         bool s_waited = it == 0;  // the peer has finished reading the previous pair's probabilities in its buffer
         const uint32_t peer_S = map_to_cta(smem_u32(Sall), rank ^ 1u);
         const uint32_t peer_Pb = map_to_cta(smem_u32(Pb), rank ^ 1u);
         const uint32_t peer_pready = map_to_cta(B.p_ready, rank ^ 1u);
         float *Smine = Sall + (size_t)rank * lay.nq_local * PSTRIDE;
-        if (mine.valid > 0) {
-            // pull this tile's latent rows of every source from HBM into L2 ahead of the producers' loads
+        // pull a tile's latent rows of every source from HBM into L2 ahead of the producers' loads
+        auto prefetch_rows = [&](const TileInfo &t_) {
             int item = 0;
             for (int which = which_lo; which < which_hi; ++which)
                 for (int sidx = 0; sidx < P.n_src[which]; ++sidx) {
@@ -639,34 +650,41 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     const int n = 2 * ((sp.d + 63) >> 6);
                     if (et >= item && et < item + n) {
                         const int i = et - item, h = i & 1;
-                        if (64 * h < mine.valid) {
-                            const int t = mine.chunk * TILE + 64 * h;
-                            const int page = a.block_table[(int64_t)seqs.id[mine.si] * a.max_pages_per_seq + t / a.page_tokens];
+                        if (64 * h < t_.valid) {
+                            const int t = t_.chunk * TILE + 64 * h;
+                            const int page = a.block_table[(int64_t)seqs.id[t_.si] * a.max_pages_per_seq + t / a.page_tokens];
                             tma_prefetch_2d(sp.tm_pool, (i >> 1) * 64, page * a.page_tokens + t % a.page_tokens);
                         }
                     }
                     item += n;
                 }
+        };
+        // eight query elements (16 B) per thread and turn: scaled, to fp32 (and to bf16 rows for the tensor op)
+        auto q_store = [&](int i, const uint4 &raw) {
+            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+            float2 f[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                f[u] = __bfloat1622float2(h2[u]);
+                f[u].x *= a.scale;
+                f[u].y *= a.scale;
+            }
+            *reinterpret_cast<float4 *>(qs + i) = make_float4(f[0].x, f[0].y, f[1].x, f[1].y);
+            *reinterpret_cast<float4 *>(qs + i + 4) = make_float4(f[2].x, f[2].y, f[3].x, f[3].y);
+            if (GMMA)
+                *reinterpret_cast<uint4 *>(qb + (i >> 6) * QBS + (i & 63)) =
+                    make_uint4(pack_bf16(f[0].x, f[0].y), pack_bf16(f[1].x, f[1].y), pack_bf16(f[2].x, f[2].y),
+                               pack_bf16(f[3].x, f[3].y));
+        };
+        if (SLAB && next_ready) {
+            epi_bar_sync();  // the queries stored during the previous pair are visible to every warp
+        } else if (mine.valid > 0) {
+            prefetch_rows(mine);
             const __nv_bfloat16 *qg =
                 reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)mine.si * hq + h_lo * group) * 64;
-            for (int i = 8 * et; i < nq_part * 64; i += 8 * 256) {  // eight elements (16 B) per thread and turn
-                const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(qg + i));
-                const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-                float2 f[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    f[u] = __bfloat1622float2(h2[u]);
-                    f[u].x *= a.scale;
-                    f[u].y *= a.scale;
-                }
-                *reinterpret_cast<float4 *>(qs + i) = make_float4(f[0].x, f[0].y, f[1].x, f[1].y);
-                *reinterpret_cast<float4 *>(qs + i + 4) = make_float4(f[2].x, f[2].y, f[3].x, f[3].y);
-                if (GMMA)
-                    *reinterpret_cast<uint4 *>(qb + (i >> 6) * QBS + (i & 63)) =
-                        make_uint4(pack_bf16(f[0].x, f[0].y), pack_bf16(f[1].x, f[1].y), pack_bf16(f[2].x, f[2].y),
-                                   pack_bf16(f[3].x, f[3].y));
-            }
+            for (int i = 8 * et; i < nq_part * 64; i += 8 * 256) q_store(i, __ldg(reinterpret_cast<const uint4 *>(qg + i)));
         }
+        next_ready = false;
         for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
             const int nj = P.n_jobs[which];
@@ -697,8 +715,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 const int m = sp.m;
                 const uint32_t buf = jc & 1u;
                 const uint32_t acc = tmem + 256u * buf + tl_addr;
+                if (SLAB) {  // one parameter block per source, filled during the cluster's first pair
+                    const int pslot = which * P.n_src[0] + job.src;
+                    s1 = fparam + (size_t)pslot * (2 * m_pad + lay.max_in);
+                    t1 = s1 + m_pad;
+                    b2 = s1 + 2 * m_pad;
+                }
                 if (job.kind == 1) {
-                    if (job.first) {
+                    if (job.first && (!SLAB || it == 0)) {
                         // this source's parameters: fetched into registers first, so that the global-memory
                         // latency overlaps the wait for the other warps
                         float ps[MAX_HID_GROUPS], pt[MAX_HID_GROUPS], pb[MAX_HID_GROUPS];
@@ -829,8 +853,37 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     }
                     epi_bar_sync();
                 }
+                uint4 qraw[2];
+                bool q_held = false;
+                if (SLAB && which == 1 && !lay.kv_split && !next_ready && nq_part <= 64) {
+                    const int np = pair + pair_stride;
+                    if (np < lay.n_pairs) {
+                        tl_next[0] = locate_tile(tix, 2 * np, seqs.n);
+                        tl_next[1] = locate_tile(tix, 2 * np + 1, seqs.n);
+                        next_ready = true;
+                        const TileInfo nm = tl_next[rank];
+                        if (nm.valid > 0) {
+                            prefetch_rows(nm);
+                            const __nv_bfloat16 *qg =
+                                reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)nm.si * hq + h_lo * group) * 64;
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                const int i = 8 * et + 2048 * u;
+                                if (i < nq_part * 64) qraw[u] = __ldg(reinterpret_cast<const uint4 *>(qg + i));
+                            }
+                            q_held = true;
+                        }
+                    }
+                }
                 mbar_wait<false, 100>(B.jfull + 8 * buf, (jc >> 1) & 1u, a.status, &abort_flag, 0x302);
                 tc_fence_after();
+                if (SLAB && q_held) {  // every warp is past this pair's scores: the query rows are free
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int i = 8 * et + 2048 * u;
+                        if (i < nq_part * 64) q_store(i, qraw[u]);
+                    }
+                }
                 if (which == 0) {
                     // K: this thread owns token `row` of this CTA's tile; columns = (head place, channel)
                     const int nh = job.nh;
@@ -1188,7 +1241,7 @@ bool encode_map(EncodeTiledFn fn, void *dst_host, const void *dev_ptr, uint64_t 
 
 inline uint32_t up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int nslot) {
+PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslots, int nslot) {
     PairLaunch l{};
     const int ks_hid = (max_m + 63) / 64;
     uint32_t o = 0;
@@ -1199,7 +1252,7 @@ PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int nslot
     l.off_part = o;
     o = up(o + (uint32_t)sizeof(TcPart), 16);
     l.off_fparam = o;
-    o = up(o + (uint32_t)(2 * ((max_m + 31) & ~31) + max_in) * 4, 16);
+    o = up(o + (uint32_t)pslots * (uint32_t)(2 * ((max_m + 31) & ~31) + max_in) * 4, 16);  // parameter blocks
     l.off_q = o;
     o = up(o + (uint32_t)nq_local * 64 * 4, 16);
     l.off_s = o;
@@ -1219,9 +1272,9 @@ PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int nslot
 uint32_t launch_bytes(const PairLaunch &l) { return l.off_bar + 8u * (2 * l.nslot + N_FIXED_BARS) + 1024u; }
 
 // ring depth that fits beside everything else (0 = does not fit)
-int pick_nslot(int nq_local, int group, int max_m, int max_in) {
+int pick_nslot(int nq_local, int group, int max_m, int max_in, int pslots) {
     for (int nslot = 10; nslot >= 3; --nslot)
-        if (launch_bytes(make_launch(nq_local, group, max_m, max_in, nslot)) <= 227u * 1024u) return nslot;
+        if (launch_bytes(make_launch(nq_local, group, max_m, max_in, pslots, nslot)) <= 227u * 1024u) return nslot;
     return 0;
 }
 
@@ -1369,12 +1422,14 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
         if (!ok || max_m == 0) continue;
         TcPart *parts = reinterpret_cast<TcPart *>(img + part_off) + (size_t)l * 7;
         TcLayerCfg &lc = tc.layer[l];
+        // hidden layers of a single chunk: every source keeps its parameter block in shared memory (see SLAB)
+        const int pslots = max_m <= 256 ? plans[l].w[0].n_src + plans[l].w[1].n_src : 1;
         const int splits[3] = {1, 2, 4};
         for (int si = 0; si < 3; ++si) {
             const int split = splits[si];
             if (cfg.n_kv_heads % split) continue;
             const int per = cfg.n_kv_heads / split;
-            bool fits = pick_nslot(per * group, group, max_m, max_in) >= 3;
+            bool fits = pick_nslot(per * group, group, max_m, max_in, pslots) >= 3;
             for (int i = 0; i < split && fits; ++i)
                 fits = build_part(plans[l], srcs, i * per, (i + 1) * per, parts[part_index(split, i)]);
             lc.split_ok[si] = fits ? 1 : 0;
@@ -1383,6 +1438,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
         lc.ok = 1;
         lc.max_m = (uint16_t)max_m;
         lc.max_in = (uint16_t)max_in;
+        lc.pslots = (uint16_t)pslots;
         any = true;
     }
     if (!any) {
@@ -1428,7 +1484,8 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     }
     const int group = a.hq / a.hkv;
     const int nq_local = a.hkv / split * group;
-    PairLaunch lay = make_launch(nq_local, group, lc.max_m, lc.max_in, pick_nslot(nq_local, group, lc.max_m, lc.max_in));
+    PairLaunch lay = make_launch(nq_local, group, lc.max_m, lc.max_in, lc.pslots,
+                                 pick_nslot(nq_local, group, lc.max_m, lc.max_in, lc.pslots));
     lay.split = split;
     lay.n_pairs = n_pairs;
     lay.kv_split = kv_split;

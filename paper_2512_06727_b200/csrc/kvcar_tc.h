@@ -46,6 +46,7 @@ struct TcLayerCfg {
     uint8_t split_ok[3];   // head splits 1, 2, 4 available
     uint16_t max_m;        // widest hidden layer among the layer's sources
     uint16_t max_in;       // widest restored row among the layer's sources
+    uint16_t pslots;       // parameter blocks kept in shared memory (one per source if every hidden layer is one chunk)
 };
 
 struct TcState {
