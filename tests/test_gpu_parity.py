@@ -187,6 +187,31 @@ def test_large_grid_runs_k_then_v_in_one_cluster():
     _check_step(p.decode_step(seqs, 0), "bf16", "fused clusters")
 
 
+@pytest.mark.parametrize("shape", ["group2_narrow", "group4_wide", "group3_odd"])
+def test_tensor_kernel_variants_walk_several_pairs(shape):
+    """The tensor-core kernel is built in four variants (query groups of more than two heads or not; hidden
+    layers of one 256-column chunk or more).  The two paper shapes take two of them; these shapes take the
+    others, with more tile pairs than clusters so that a cluster walks several pairs (queries and tile
+    positions of the next pair fetched ahead, parameter blocks kept, probability buffers handed back)."""
+    if shape == "group2_narrow":     # 8 query / 4 KV heads, hidden 192: one chunk, CUDA-core attention products
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, n_q_heads=8, n_kv_heads=4, latent_full=128, batch=9,
+                         cached_tokens=0, decode_steps=1, reuse_frac=0.25)
+    elif shape == "group4_wide":     # 32 query / 8 KV heads, hidden 384: two chunks, tensor-op attention products
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, n_q_heads=32, n_kv_heads=8, latent_full=256, batch=9,
+                         cached_tokens=0, decode_steps=1, reuse_frac=0.25)
+    else:                            # 6 query / 2 KV heads: a group of three (padded inside the 8-wide operand)
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, n_q_heads=6, n_kv_heads=2, latent_full=64, batch=9,
+                         cached_tokens=0, decode_steps=1, reuse_frac=0.5)
+    pps = 34
+    p = Pair(w, max_seqs=9, max_pages=9 * pps, max_pages_per_seq=pps, kernel=B.KERNEL_TENSOR)
+    seqs = list(range(9))
+    p.open(seqs)
+    for s_, n in zip(seqs, (2100, 2049, 2111, 2050, 2064, 2051, 2172, 2090, 2055)):   # 17 tiles each: 77 pairs
+        p.prefill([s_], n)
+    assert all(p.s.ctx.layer_kernel(l) == B.KERNEL_TENSOR for l in range(w.n_layers))
+    _check_step(p.decode_step(seqs, 0), "bf16", shape)
+
+
 def test_fp32_stack_with_reuse_generic():
     """fp32 mode on a multi-layer stack with chains of reuse; 1e-4 absolute."""
     w = synth.scaled(synth.CONFIGS["c2"], n_layers=4, batch=2, storage="f32", reuse_frac=0.5)
