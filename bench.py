@@ -48,6 +48,9 @@ def parse():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tensor"])
     ap.add_argument("--uncompressed", action="store_true", help="raw K/V pages (the uncompressed twin)")
+    ap.add_argument("--api", default="fused", choices=["fused", "split"],
+                    help="a layer's step through kvcar_step_layer (one call; the tile kernel runs beside the encoder) "
+                         "or through kvcar_encode_append + kvcar_decode_attention")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle sample")
@@ -189,11 +192,15 @@ def step_inputs(sess, w, torch, n_steps):
     return k, v, q, out
 
 
-def run_step(sess, w, seqs, k, v, q, out, i, stream, flags):
+def run_step(sess, w, seqs, k, v, q, out, i, stream, flags, fused=True):
     ctx = sess.ctx
     for l in range(w.n_layers):
-        ctx.encode_append(l, seqs, 1, k[i, l].data_ptr(), v[i, l].data_ptr(), stream)
-        ctx.decode_attention(l, seqs, q[i, l].data_ptr(), out[i, l].data_ptr(), flags, stream)
+        if fused:
+            ctx.step_layer(l, seqs, k[i, l].data_ptr(), v[i, l].data_ptr(), q[i, l].data_ptr(), out[i, l].data_ptr(),
+                           flags, stream)
+        else:
+            ctx.encode_append(l, seqs, 1, k[i, l].data_ptr(), v[i, l].data_ptr(), stream)
+            ctx.decode_attention(l, seqs, q[i, l].data_ptr(), out[i, l].data_ptr(), flags, stream)
     ctx.advance(seqs, 1, stream)
 
 
@@ -376,8 +383,9 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()          # nvidia-smi needs a moment to come up: it samples warm-up, timed region and pass 2
+    fused = args.api == "fused"
     for i in range(W_):
-        run_step(sess, w, seqs, k, v, q, out, i, stream, flags)
+        run_step(sess, w, seqs, k, v, q, out, i, stream, flags, fused)
     sess.ctx.sync_status(stream)
     launches0 = sess.ctx.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_)]
@@ -386,7 +394,7 @@ def main():
     for j in range(K_):
         flush.fill_(j & 0xFF)                      # evict the cache from L2 between steps (outside the event pair)
         ev[j][0].record()
-        run_step(sess, w, seqs, k, v, q, out, W_ + j, stream, flags)
+        run_step(sess, w, seqs, k, v, q, out, W_ + j, stream, flags, fused)
         ev[j][1].record()
     barrier()
     wall = time.perf_counter() - wall0
@@ -496,7 +504,7 @@ def main():
                 "config": {"workload": w.name, "batch_per_gpu": w.batch, "cached_tokens": w.cached_tokens,
                            "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
                            "latent_full": 0 if args.uncompressed else w.latent_full, "reuse_frac": w.reuse_frac,
-                           "page_tokens": w.page_tokens, "kernel": args.kernel,
+                           "page_tokens": w.page_tokens, "kernel": args.kernel, "api": args.api,
                            "uncompressed": bool(args.uncompressed),
                            "l2": "flushed between steps (256 MiB write outside the per-step event pairs)",
                            "cache_bytes_per_token": comp, "uncompressed_bytes_per_token": full,

@@ -192,9 +192,25 @@ kvcar_status kvcar_decode_attention(kvcar_ctx *ctx, int32_t layer, const int32_t
                                     const void *q, void *out, uint32_t flags, void *stream);
 
 /*
- * The same two calls for one layer with HOST buffers: copies k, v, q (each
- * n_tokens = 1) to the device, runs kvcar_encode_append then
- * kvcar_decode_attention, and copies `out` back, all on `stream`.  Returns
+ * One decode step of one layer in one call: kvcar_encode_append (n_tokens = 1)
+ * of k, v followed by kvcar_decode_attention of q, same arguments, same
+ * results, all DEVICE buffers.  Because the cached rows that the decoder reads
+ * do not depend on the row the encoder appends (Sec. "Network Architecture":
+ * the restored (l-1) x D matrices are concatenated with the current token's
+ * exact vectors, which enter only when the tiles are merged), the library runs
+ * the tile kernel on a stream of its own, forked from `stream` at the call and
+ * joined back before the merge, beside the encoder's launches.  On return all
+ * work is enqueued and ordered after what `stream` held at the call and before
+ * what is enqueued on it afterwards.
+ * Errors as for the two calls; on KVCAR_ERR_OOM_PAGES nothing is written.
+ */
+kvcar_status kvcar_step_layer(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *k,
+                              const void *v, const void *q, void *out, uint32_t flags, void *stream);
+
+/*
+ * The same step for one layer with HOST buffers: copies k, v, q (each
+ * n_tokens = 1) to the device, runs kvcar_step_layer, and copies `out`
+ * back, all ordered on `stream`.  Returns
  * after enqueuing; synchronise the stream before reading out_host.  Host
  * buffers should be page-locked for the copies to be asynchronous.
  */

@@ -27,7 +27,7 @@ EXPORTS = [
     "kvcar_create", "kvcar_destroy", "kvcar_set_reuse_map", "kvcar_set_autoencoder", "kvcar_required_bytes",
     "kvcar_bind_memory", "kvcar_set_kernel", "kvcar_seq_open", "kvcar_seq_close", "kvcar_reserve",
     "kvcar_encode_append", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
-    "kvcar_step_layer_host",
+    "kvcar_step_layer", "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
     "kvcar_last_error",
@@ -83,6 +83,7 @@ def load() -> C.CDLL:
         "kvcar_advance": [vp, ip, i32, i32, vp],
         "kvcar_decode_attention": [vp, i32, ip, i32, vp, vp, u32, vp],
         "kvcar_decode_attention_static": [vp, i32, ip, i32, vp, vp, u32, vp],
+        "kvcar_step_layer": [vp, i32, ip, i32, vp, vp, vp, vp, u32, vp],
         "kvcar_step_layer_host": [vp, i32, ip, i32, vp, vp, vp, vp, u32, vp],
         "kvcar_debug_resolve": [vp, i32, i32, i32, ip, ip, ip],
         "kvcar_debug_locate": [vp, i32, i32, ip, C.POINTER(C.c_int64)],
@@ -215,6 +216,11 @@ class Context:
         (allocates nothing; see kvcar_decode_attention_static in kvcar.h)."""
         self._check(self.lib.kvcar_decode_attention_static(self._h, layer, self._seqs(seqs), len(seqs), q, out,
                                                            flags, stream))
+
+    def step_layer(self, layer: int, seqs: Sequence[int], k: int, v: int, q: int, out: int,
+                   flags: int = INCLUDE_CURRENT_EXACT, stream: int = 0):
+        """encode_append (one token) + decode_attention of one layer in one call, device buffers."""
+        self._check(self.lib.kvcar_step_layer(self._h, layer, self._seqs(seqs), len(seqs), k, v, q, out, flags, stream))
 
     def step_layer_host(self, layer: int, seqs: Sequence[int], k_host: int, v_host: int, q_host: int,
                         out_host: int, flags: int = INCLUDE_CURRENT_EXACT, stream: int = 0):

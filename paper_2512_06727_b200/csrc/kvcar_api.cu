@@ -37,6 +37,9 @@ struct kvcar_ctx {
     std::vector<AEHost> ae;  // [layer*2 + which]
     bool bound = false;
     int kernel = KVCAR_KERNEL_AUTO;
+    // kvcar_step_layer runs the tile kernel beside the encoder: a stream and two events of the library's own
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 
     // pages
     std::vector<int32_t> free_pages;
@@ -312,6 +315,9 @@ kvcar_status kvcar_create(const kvcar_config *cfg, kvcar_ctx **out_ctx) {
 kvcar_status kvcar_destroy(kvcar_ctx *ctx) {
     if (!ctx) return KVCAR_ERR_INVALID_ARG;
     tc_destroy(ctx->tc);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     delete ctx;
     return KVCAR_OK;
 }
@@ -531,6 +537,15 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->kvsplit_off, 0, tc_split_bytes(g), st);  // hand-over flags
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(c, e, "upload of packed weights");
+    if (!c->side) {  // for kvcar_step_layer; without them it runs its launches in order on the caller's stream
+        if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            if (c->side) cudaStreamDestroy(c->side);
+            c->side = nullptr;
+        }
+    }
     c->bound = true;
     c->pending.clear();
     // re-queue what host bookkeeping already holds (sequences opened / pages reserved before binding)
@@ -575,6 +590,9 @@ kvcar_status kvcar_reserve(kvcar_ctx *c, const int32_t *seqs, int32_t n_seqs, in
     return reserve_pages(c, seqs, n_seqs, n_tokens);
 }
 
+static kvcar_status enqueue_encode(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens,
+                                   const void *k, const void *v, cudaStream_t st);
+
 kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens,
                                  const void *k, const void *v, void *stream) {
     if (!c) return KVCAR_ERR_INVALID_ARG;
@@ -588,6 +606,12 @@ kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seq
     cudaStream_t st = (cudaStream_t)stream;
     s = flush_tables(c, st);
     if (s != KVCAR_OK) return s;
+    return enqueue_encode(c, layer, seqs, n_seqs, n_tokens, k, v, st);
+}
+
+// the encoder launches of one layer (arguments checked, pages reserved and tables flushed by the caller)
+static kvcar_status enqueue_encode(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens,
+                                   const void *k, const void *v, cudaStream_t st) {
     EncodeArgs a{};
     a.plan = reinterpret_cast<const EncPlan *>(c->weights + c->enc_off) + layer * 2;
     a.block_table = reinterpret_cast<const int32_t *>(c->ws + c->bt_off);
@@ -634,22 +658,13 @@ kvcar_status kvcar_advance(kvcar_ctx *c, const int32_t *seqs, int32_t n_seqs, in
     return KVCAR_OK;
 }
 
-kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *q,
-                                    void *out, uint32_t flags, void *stream) {
-    if (!c) return KVCAR_ERR_INVALID_ARG;
-    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
-    if (layer < 0 || layer >= c->cfg.n_layers || !q || !out)
-        return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
-    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
-    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
-    if (flags & ~KVCAR_INCLUDE_CURRENT_EXACT) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
-    cudaStream_t st = (cudaStream_t)stream;
-    kvcar_status s = flush_tables(c, st);
-    if (s != KVCAR_OK) return s;
+// launch arguments of one layer's decode; returns the number of tiles along the longest listed sequence
+static int prepare_decode(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *q, void *out,
+                          uint32_t flags, DecodeArgs &a, SeqList &sl) {
     const kvcar_config &g = c->cfg;
     int max_len = 0;
     for (int i = 0; i < n_seqs; ++i) max_len = std::max(max_len, c->len[seqs[i]]);
-    DecodeArgs a{};
+    a = DecodeArgs{};
     a.plan = reinterpret_cast<const LayerPlan *>(c->weights + c->plan_off) + layer;
     a.block_table = reinterpret_cast<const int32_t *>(c->ws + c->bt_off);
     a.seq_len = reinterpret_cast<const int32_t *>(c->ws + c->len_off);
@@ -666,33 +681,115 @@ kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *
     a.max_chunks = c->max_chunks;
     a.flags = flags;
     a.scale = 1.0f / std::sqrt((float)g.head_dim);
-    SeqList sl;
     sl.n = n_seqs;
     memcpy(sl.id, seqs, (size_t)n_seqs * 4);
-    const int n_chunks = (max_len + c->chunk_tokens - 1) / c->chunk_tokens;
-    if (n_chunks > 0) {
-        const bool want_tc = use_tensor_kernel(c) && tc_layer_supported(c->tc, layer);
-        if (c->kernel == KVCAR_KERNEL_TENSOR && !want_tc)
-            return fail(c, KVCAR_ERR_UNSUPPORTED, std::string("tensor-core kernel cannot run this layer: ") + c->tc.why);
-        cudaError_t e;
-        if (c->kernel != KVCAR_KERNEL_GENERIC && layer_is_raw(c, layer)) {
-            e = launch_decode_raw(a, sl, g.storage, n_chunks, st);
-        } else if (want_tc) {
-            int32_t lens[KVCAR_MAX_BATCH];
-            for (int i = 0; i < n_seqs; ++i) lens[i] = c->len[seqs[i]];
-            e = tc_launch_decode(c->tc, a, sl, lens, layer, st);
-        } else {
-            if (decode_generic_smem(a.hq, a.hd, c->max_d, c->max_m) > 227 * 1024)
-                return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");
-            e = launch_decode_generic(a, sl, g.storage, c->max_d, c->max_m, n_chunks, st);
-        }
-        if (e != cudaSuccess) return cuda_fail(c, e, "decode launch");
-        ++c->launches;
+    return (max_len + c->chunk_tokens - 1) / c->chunk_tokens;
+}
+
+// The kernel that works through the cached tokens tile by tile (tensor-core, raw or generic) and leaves one partial
+// result per tile.  It reads the cache rows below the sequences' lengths, the tables and q - nothing that this
+// step's encoder writes (the exact current token enters in the combine kernel).
+static kvcar_status enqueue_decode_tiles(kvcar_ctx *c, int32_t layer, const DecodeArgs &a, const SeqList &sl,
+                                         int n_chunks, cudaStream_t st) {
+    if (n_chunks <= 0) return KVCAR_OK;
+    const kvcar_config &g = c->cfg;
+    const bool want_tc = use_tensor_kernel(c) && tc_layer_supported(c->tc, layer);
+    if (c->kernel == KVCAR_KERNEL_TENSOR && !want_tc)
+        return fail(c, KVCAR_ERR_UNSUPPORTED, std::string("tensor-core kernel cannot run this layer: ") + c->tc.why);
+    cudaError_t e;
+    if (c->kernel != KVCAR_KERNEL_GENERIC && layer_is_raw(c, layer)) {
+        e = launch_decode_raw(a, sl, g.storage, n_chunks, st);
+    } else if (want_tc) {
+        int32_t lens[KVCAR_MAX_BATCH];
+        for (int i = 0; i < sl.n; ++i) lens[i] = c->len[sl.id[i]];
+        e = tc_launch_decode(c->tc, a, sl, lens, layer, st);
+    } else {
+        if (decode_generic_smem(a.hq, a.hd, c->max_d, c->max_m) > 227 * 1024)
+            return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");
+        e = launch_decode_generic(a, sl, g.storage, c->max_d, c->max_m, n_chunks, st);
     }
-    cudaError_t e = launch_combine(a, sl, g.storage, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "decode launch");
+    ++c->launches;
+    return KVCAR_OK;
+}
+
+static kvcar_status enqueue_combine(kvcar_ctx *c, const DecodeArgs &a, const SeqList &sl, cudaStream_t st) {
+    cudaError_t e = launch_combine(a, sl, c->cfg.storage, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "combine launch");
     ++c->launches;
     return KVCAR_OK;
+}
+
+static kvcar_status check_decode_args(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *q,
+                                      const void *out, uint32_t flags) {
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (layer < 0 || layer >= c->cfg.n_layers || !q || !out)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
+    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    if (flags & ~KVCAR_INCLUDE_CURRENT_EXACT) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *q,
+                                    void *out, uint32_t flags, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    kvcar_status s = check_decode_args(c, layer, seqs, n_seqs, q, out, flags);
+    if (s != KVCAR_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    s = flush_tables(c, st);
+    if (s != KVCAR_OK) return s;
+    DecodeArgs a;
+    SeqList sl;
+    const int n_chunks = prepare_decode(c, layer, seqs, n_seqs, q, out, flags, a, sl);
+    s = enqueue_decode_tiles(c, layer, a, sl, n_chunks, st);
+    if (s != KVCAR_OK) return s;
+    return enqueue_combine(c, a, sl, st);
+}
+
+kvcar_status kvcar_step_layer(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *k,
+                              const void *v, const void *q, void *out, uint32_t flags, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    kvcar_status s = check_decode_args(c, layer, seqs, n_seqs, q, out, flags);
+    if (s != KVCAR_OK) return s;
+    if (!k || !v) return fail(c, KVCAR_ERR_INVALID_ARG, "null k or v");
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "k/v must be 16-byte aligned");
+    s = reserve_pages(c, seqs, n_seqs, 1);
+    if (s != KVCAR_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    s = flush_tables(c, st);
+    if (s != KVCAR_OK) return s;
+    DecodeArgs a;
+    SeqList sl;
+    const int n_chunks = prepare_decode(c, layer, seqs, n_seqs, q, out, flags, a, sl);
+    // The tile kernel does not depend on this step's encoder, so it goes to a side stream that forks here and
+    // joins before the combine kernel: the encoder's two small launches run beside it (on the SMs a small grid
+    // leaves idle, or in its shadow) instead of in front of it.  The tile kernel is enqueued first so that it
+    // is placed first.
+    const bool fork = c->side != nullptr && n_chunks > 0;
+    if (fork) {
+        cudaError_t e = cudaEventRecord(c->ev_fork, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e, "stream fork");
+        s = enqueue_decode_tiles(c, layer, a, sl, n_chunks, c->side);
+        cudaError_t e2 = cudaEventRecord(c->ev_join, c->side);  // recorded even after a failed launch: the join below
+        if (s != KVCAR_OK) {                                     // must not leave the side stream detached
+            cudaStreamWaitEvent(st, c->ev_join, 0);
+            return s;
+        }
+        if (e2 != cudaSuccess) return cuda_fail(c, e2, "stream join");
+    }
+    s = enqueue_encode(c, layer, seqs, n_seqs, 1, k, v, st);
+    if (fork) {
+        cudaError_t e = cudaStreamWaitEvent(st, c->ev_join, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e, "stream join");
+    }
+    if (s != KVCAR_OK) return s;
+    if (!fork) {
+        s = enqueue_decode_tiles(c, layer, a, sl, n_chunks, st);
+        if (s != KVCAR_OK) return s;
+    }
+    return enqueue_combine(c, a, sl, st);
 }
 
 kvcar_status kvcar_step_layer_host(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs,
@@ -714,9 +811,7 @@ kvcar_status kvcar_step_layer_host(kvcar_ctx *c, int32_t layer, const int32_t *s
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(dq, q_host, (size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "host to device copy");
-    kvcar_status s = kvcar_encode_append(c, layer, seqs, n_seqs, 1, dk, dv, stream);
-    if (s != KVCAR_OK) return s;
-    s = kvcar_decode_attention(c, layer, seqs, n_seqs, dq, dout, flags, stream);
+    kvcar_status s = kvcar_step_layer(c, layer, seqs, n_seqs, dk, dv, dq, dout, flags, stream);
     if (s != KVCAR_OK) return s;
     e = cudaMemcpyAsync(out_host, dout, (size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "device to host copy");

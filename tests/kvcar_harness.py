@@ -113,16 +113,40 @@ class Pair:
                 ref = self.o.decode_attention(layer, [seqs[i] for i in rows], q[rows], include_current=include_current)
         return got, ref, rows
 
+    def step_layer(self, layer: int, seqs: Sequence[int], k: np.ndarray, v: np.ndarray, q: np.ndarray,
+                   include_current: bool = True):
+        """append + attention of one layer through the single-call entry point; same return as attention()."""
+        dk, dv, dq = self.s.to_device(k), self.s.to_device(v), self.s.to_device(q)
+        out = torch.empty_like(dq)
+        flags = B.INCLUDE_CURRENT_EXACT if include_current else 0
+        self.s.ctx.step_layer(layer, list(seqs), dk.data_ptr(), dv.data_ptr(), dq.data_ptr(), out.data_ptr(), flags,
+                              self.s.stream())
+        self.s.ctx.sync_status(self.s.stream())
+        got = out.float().cpu().numpy().astype(np.float64)
+        ref, rows = None, []
+        if self.o is not None:
+            rows = self._oracle_rows(seqs)
+            if rows:
+                sub = [seqs[i] for i in rows]
+                self.o.encode_append(layer, sub, 1, k[rows], v[rows])
+                ref = self.o.decode_attention(layer, sub, q[rows], include_current=include_current)
+        return got, ref, rows
+
     def decode_step(self, seqs: Sequence[int], step: int, q_scale: float = 1.0, include_current: bool = True,
-                    layers: Optional[Sequence[int]] = None):
+                    layers: Optional[Sequence[int]] = None, fused: bool = False):
         """One full decode step (encode-append + attention for every layer, then
-        advance).  Returns per-layer (gpu, oracle, rows)."""
+        advance).  Returns per-layer (gpu, oracle, rows).  fused: each layer through
+        the single-call entry point instead of the two calls."""
         w = self.w
         res = {}
         t = {s: self.s.ctx.seq_len(s) for s in seqs}
         for l in range(w.n_layers):
             k = np.stack([synth.make_kv(w, l, K, s, t[s], 1) for s in seqs])
             v = np.stack([synth.make_kv(w, l, V, s, t[s], 1) for s in seqs])
+            if fused:
+                q = np.stack([synth.make_q(w, l, s, step, scale=q_scale) for s in seqs])
+                res[l] = self.step_layer(l, seqs, k, v, q, include_current)
+                continue
             self.append(l, seqs, k, v)
             if layers is None or l in layers:
                 q = np.stack([synth.make_q(w, l, s, step, scale=q_scale) for s in seqs])

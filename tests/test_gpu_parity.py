@@ -224,6 +224,30 @@ def test_fp32_stack_with_reuse_generic():
         _check_step(p.decode_step([0, 1], step), "f32", f"step {step}")
 
 
+@pytest.mark.parametrize("cfg", ["c2", "c3"])
+def test_single_call_step_matches_oracle_and_the_two_calls(cfg):
+    """kvcar_step_layer (tile kernel on the library's side stream beside the encoder) against the oracle, and bit
+    for bit against kvcar_encode_append + kvcar_decode_attention on a twin context, over several steps (so that
+    later steps read rows appended by earlier ones) and a page boundary."""
+    w = synth.scaled(synth.CONFIGS[cfg], n_layers=4, batch=3, cached_tokens=0, decode_steps=3, reuse_frac=0.3)
+    seqs = [0, 1, 2]
+    pairs = []
+    for with_oracle in (True, False):
+        p = Pair(w, max_seqs=3, max_pages=24, max_pages_per_seq=8, with_oracle=with_oracle)
+        p.open(seqs)
+        for s_, n in zip(seqs, (383, 130, 62)):        # the third sequence crosses a page boundary at step 2
+            p.prefill([s_], n)
+        pairs.append(p)
+    fused, split = pairs
+    for step in range(3):
+        a = fused.decode_step(seqs, step, fused=True)
+        b = split.decode_step(seqs, step, fused=False)
+        _check_step(a, "bf16", f"single call, step {step}")
+        for l in a:
+            assert np.array_equal(a[l][0], b[l][0]), (step, l)
+    fused.check_latents(seqs)
+
+
 def test_host_buffer_entry_point_matches_device_entry_points():
     w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=2, reuse_frac=0.25)
     p = Pair(w, max_seqs=2, max_pages=8, max_pages_per_seq=4)
