@@ -363,47 +363,84 @@ __global__ void __launch_bounds__(NT) decode_generic_kernel(const __grid_constan
 }
 
 // ---------------------------------------------------------------------------
-// Combine the chunk partials of one (sequence, query head) and, if asked, the
-// exact current token.  grid = (hq, n_seqs); block = 128 (threads >= hd idle).
+// Combine the tile partials of one (sequence, query head) and, if asked, the
+// exact current token.  grid = (hq, n_seqs); block = 256.  A long sequence has
+// hundreds of tiles, so nothing walks them one after the other: three passes of
+// independent loads (largest maximum; sum of the sums scaled to it; weighted
+// values, one warp per tile in turns, lanes over the channels), each closed by a
+// block reduction.
+constexpr int CB_WARPS = 8;
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float *red) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float u = __shfl_xor_sync(0xffffffffu, v, o);
+        v = is_max ? fmaxf(v, u) : v + u;
+    }
+    __syncthreads();  // red may still be read from the previous reduction
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    v = red[0];
+#pragma unroll
+    for (int w = 1; w < CB_WARPS; ++w) v = is_max ? fmaxf(v, red[w]) : v + red[w];
+    return v;
+}
+
 template <typename T>
-__global__ void __launch_bounds__(128) combine_kernel(const __grid_constant__ DecodeArgs a,
-                                                      const __grid_constant__ SeqList seqs) {
-    const int qh = blockIdx.x, si = blockIdx.y, c = threadIdx.x;
+__global__ void __launch_bounds__(32 * CB_WARPS) combine_kernel(const __grid_constant__ DecodeArgs a,
+                                                                const __grid_constant__ SeqList seqs) {
+    const int qh = blockIdx.x, si = blockIdx.y, c = threadIdx.x, lane = c & 31, warp = c >> 5;
     const int seq = seqs.id[si];
     const int L = a.seq_len[seq];
-    const int hd = a.hd, hq = a.hq;
+    const int hd = a.hd, hq = a.hq;  // hd <= 128
     const int n_chunks = (L + a.chunk_tokens - 1) / a.chunk_tokens;
     const bool on = c < hd;
-    float M = -INFINITY, S = 0.f, acc = 0.f;
-    for (int ch = 0; ch < n_chunks; ++ch) {
-        const float *part = a.partials + (((int64_t)si * a.max_chunks + ch) * hq + qh) * (hd + 2);
-        float m = part[0], s = part[1];
-        float v = on ? part[2 + c] : 0.f;
-        float Mn = fmaxf(M, m);
-        float c0 = (M == -INFINITY) ? 0.f : expf(M - Mn);
-        float c1 = (m == -INFINITY) ? 0.f : expf(m - Mn);
-        S = S * c0 + s * c1;
-        acc = acc * c0 + v * c1;
-        M = Mn;
+    const int64_t stride = (int64_t)hq * (hd + 2);  // floats from one tile's partial to the next
+    const float *base = a.partials + ((int64_t)si * a.max_chunks * hq + qh) * (hd + 2);
+    __shared__ float red[CB_WARPS];
+    __shared__ float accs[CB_WARPS][128];
+
+    float M = -INFINITY;
+    for (int ch = c; ch < n_chunks; ch += 32 * CB_WARPS) M = fmaxf(M, base[ch * stride]);
+    M = block_reduce(M, true, red);
+    float S = 0.f;
+    for (int ch = c; ch < n_chunks; ch += 32 * CB_WARPS) {
+        const float m = base[ch * stride], s = base[ch * stride + 1];
+        S += (m == -INFINITY) ? 0.f : s * expf(m - M);
     }
+    S = block_reduce(S, false, red);
+    float av[4] = {0.f, 0.f, 0.f, 0.f};  // channels lane, lane + 32, lane + 64, lane + 96
+#pragma unroll 4
+    for (int ch = warp; ch < n_chunks; ch += CB_WARPS) {
+        const float *part = base + ch * stride;
+        const float m = part[0];
+        const float w = (m == -INFINITY) ? 0.f : expf(m - M);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (lane + 32 * j < hd) av[j] = fmaf(w, part[2 + lane + 32 * j], av[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) accs[warp][lane + 32 * j] = av[j];
+    __syncthreads();
+    float acc = 0.f;
+    if (on)
+#pragma unroll
+        for (int w = 0; w < CB_WARPS; ++w) acc += accs[w][c];
+
     if (a.flags & KVCAR_INCLUDE_CURRENT_EXACT) {
         const int g = qh / (hq / a.hkv);
         const int W = a.hkv * hd;
         const T *kc = reinterpret_cast<const T *>(a.plan->cur[0][g]) + (int64_t)seq * W + a.plan->cur_head[0][g] * hd;
         const T *vc = reinterpret_cast<const T *>(a.plan->cur[1][g]) + (int64_t)seq * W + a.plan->cur_head[1][g] * hd;
         const T *qg = reinterpret_cast<const T *>(a.q) + ((int64_t)si * hq + qh) * hd;
-        __shared__ float red[4];
-        float prod = on ? ld(qg + c) * ld(kc + c) : 0.f;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) prod += __shfl_xor_sync(0xffffffffu, prod, o);
-        if ((c & 31) == 0) red[c >> 5] = prod;
-        __syncthreads();
-        float sc = (red[0] + red[1] + red[2] + red[3]) * a.scale;
-        float Mn = fmaxf(M, sc);
-        float c0 = (M == -INFINITY) ? 0.f : expf(M - Mn);
-        float c1 = expf(sc - Mn);
+        const float vcur = on ? ld(vc + c) : 0.f;
+        const float sc = block_reduce(on ? ld(qg + c) * ld(kc + c) : 0.f, false, red) * a.scale;
+        const float Mn = fmaxf(M, sc);
+        const float c0 = (M == -INFINITY) ? 0.f : expf(M - Mn);
+        const float c1 = expf(sc - Mn);
         S = S * c0 + c1;
-        acc = acc * c0 + (on ? ld(vc + c) : 0.f) * c1;
+        acc = acc * c0 + vcur * c1;
     }
     if (on) {
         T *o = reinterpret_cast<T *>(a.out) + ((int64_t)si * hq + qh) * hd;
@@ -463,9 +500,9 @@ cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int 
 cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, cudaStream_t st) {
     dim3 grid(a.hq, seqs.n);
     if (dtype == KVCAR_F32)
-        combine_kernel<float><<<grid, 128, 0, st>>>(a, seqs);
+        combine_kernel<float><<<grid, 32 * CB_WARPS, 0, st>>>(a, seqs);
     else
-        combine_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>(a, seqs);
+        combine_kernel<__nv_bfloat16><<<grid, 32 * CB_WARPS, 0, st>>>(a, seqs);
     return cudaGetLastError();
 }
 
