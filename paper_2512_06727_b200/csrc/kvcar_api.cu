@@ -763,9 +763,9 @@ kvcar_status kvcar_step_layer(kvcar_ctx *c, int32_t layer, const int32_t *seqs, 
     SeqList sl;
     const int n_chunks = prepare_decode(c, layer, seqs, n_seqs, q, out, flags, a, sl);
     // The tile kernel does not depend on this step's encoder, so it goes to a side stream that forks here and
-    // joins before the combine kernel: the encoder's two small launches run beside it (on the SMs a small grid
-    // leaves idle, or in its shadow) instead of in front of it.  The tile kernel is enqueued first so that it
-    // is placed first.
+    // joins before the combine kernel: the encoder's two short launches overlap it instead of running in front
+    // of it.  (The other way round - encoder on the side stream behind the fork event - measured no gain: the
+    // encoder then finds a small grid's few idle SMs only and outlasts the tile kernel.)
     const bool fork = c->side != nullptr && n_chunks > 0;
     if (fork) {
         cudaError_t e = cudaEventRecord(c->ev_fork, st);
