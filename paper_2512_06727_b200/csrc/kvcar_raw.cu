@@ -193,10 +193,193 @@ __global__ void __launch_bounds__(RW * 32, 4) decode_raw_kernel(const __grid_con
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Query groups of more than two heads, bf16 rows: the dots of a group against a row are a small matrix product,
+// and on the CUDA cores they, not HBM, set the pace (8 heads: 1024 FMA per cached row and KV head).  Same
+// decomposition (one warp per sequence, 128-token tile and KV head), but 32 tokens at a time go through shared
+// memory (cp.async, 16-byte chunks swizzled by row, the next 32 tokens in flight meanwhile) into the warp-level
+// tensor op: scores^T[8 queries x 8 tokens] = Q . K^T with the K rows as the "column-major" operand they already
+// are; the probabilities come out in the layout the next product wants as its row operand (queries x tokens), and
+// V enters through transposing matrix loads.  Online softmax across the four 32-token steps, fp32.
+constexpr int GQ_STEP = 32;                      // tokens per step
+constexpr int GQ_BUF = GQ_STEP * 64 * 2;         // bytes of one K (or V) step buffer: 32 rows x 128 B
+constexpr int GQ_WARP_SMEM = 4 * GQ_BUF;         // K and V, two steps each
+constexpr int GQ_SMEM = RW * GQ_WARP_SMEM;
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t *r) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t *r) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D[16 x 8] += A[16 x 16] . B[16 x 8], bf16 in, fp32 out; rows 8..15 of A are zero here (a1 = a3 = 0)
+__device__ __forceinline__ void mma_q8(float *d, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %5}, {%7, %8}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+__global__ void __launch_bounds__(RW * 32) decode_raw_gq_kernel(const __grid_constant__ DecodeArgs a,
+                                                               const __grid_constant__ SeqList seqs) {
+    extern __shared__ __align__(128) uint8_t gq_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x, h = blockIdx.y * RW + warp, si = blockIdx.z;
+    if (h >= a.hkv) return;
+    const int seq = seqs.id[si];
+    const int L = a.seq_len[seq];
+    const int t0 = tile * RT;
+    if (t0 >= L) return;
+    const int valid = min(RT, L - t0);
+    const int group = a.hq / a.hkv;
+    const HeadSrc ks = find_head(a.plan->w[0], h), vs = find_head(a.plan->w[1], h);
+    const __nv_bfloat16 *kpool = reinterpret_cast<const __nv_bfloat16 *>(ks.pool) + ks.col;
+    const __nv_bfloat16 *vpool = reinterpret_cast<const __nv_bfloat16 *>(vs.pool) + vs.col;
+    const int32_t *bt = a.block_table + (int64_t)seq * a.max_pages_per_seq;
+    const uint32_t sbase = smem_addr(gq_smem) + warp * GQ_WARP_SMEM;  // K step buffers 0, 1, then V step buffers 0, 1
+    const int g = lane >> 2, t = lane & 3;
+
+    // this lane's part of the row operand Q[16 x 64] (rows >= group are zero): per 16-channel step, channels
+    // 2t, 2t+1 and 2t+8, 2t+9 of query g
+    uint32_t qa[4][2];
+    {
+        const __nv_bfloat16 *qg = reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)si * a.hq + h * group + g) * 64;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            qa[k][0] = g < group ? __ldg(reinterpret_cast<const uint32_t *>(qg + 16 * k + 2 * t)) : 0u;
+            qa[k][1] = g < group ? __ldg(reinterpret_cast<const uint32_t *>(qg + 16 * k + 8 + 2 * t)) : 0u;
+        }
+    }
+    // fetch one 32-token step: lane = (row within a group of four, 16-byte chunk); rows past the tile's end re-read
+    // the tile's first row (their probabilities are zero)
+    auto fetch = [&](int step, int buf) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = 4 * i + (lane >> 3), c = lane & 7;
+            int tok = t0 + GQ_STEP * step + r;
+            if (tok >= t0 + valid) tok = t0;
+            const int64_t row = (int64_t)bt[tok / a.page_tokens] * a.page_tokens + tok % a.page_tokens;
+            const uint32_t off = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+            cp_async16(sbase + buf * GQ_BUF + off, kpool + row * ks.width + 8 * c);
+            cp_async16(sbase + (2 + buf) * GQ_BUF + off, vpool + row * vs.width + 8 * c);
+        }
+        cp_async_commit();
+    };
+
+    float m_run = -INFINITY, l_run = 0.f;  // of query g (the four lanes of a group hold copies)
+    float o[8][4];                         // o[n][0..1]: query g, channels 8n + 2t, 8n + 2t + 1
+#pragma unroll
+    for (int n = 0; n < 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+    const int n_steps = (valid + GQ_STEP - 1) / GQ_STEP;
+    fetch(0, 0);
+    for (int step = 0; step < n_steps; ++step) {
+        const int buf = step & 1;
+        if (step + 1 < n_steps) {
+            fetch(step + 1, buf ^ 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncwarp();
+        const uint32_t kb = sbase + buf * GQ_BUF, vb = sbase + (2 + buf) * GQ_BUF;
+        // scores^T: four blocks of 8 tokens; sc[nt][0..1] = query g, tokens 8 nt + 2t, + 1
+        float sc[4][4];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+            const int r = 8 * nt + (lane & 7);
+#pragma unroll
+            for (int kp = 0; kp < 2; ++kp) {  // two 16-channel steps per matrix load
+                uint32_t b[4];
+                ldmatrix_x4(kb + r * 128 + (((4 * kp + (lane >> 3)) ^ (r & 7)) << 4), b);
+                mma_q8(sc[nt], qa[2 * kp][0], qa[2 * kp][1], b[0], b[1]);
+                mma_q8(sc[nt], qa[2 * kp + 1][0], qa[2 * kp + 1][1], b[2], b[3]);
+            }
+        }
+        // online softmax of query g over this step's 32 tokens
+        float mx = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int tok = GQ_STEP * step + 8 * nt + 2 * t + e;
+                sc[nt][e] = tok < valid ? sc[nt][e] * a.scale : -INFINITY;
+                mx = fmaxf(mx, sc[nt][e]);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);  // finite: the step holds at least one valid token
+        const float corr = m_run == -INFINITY ? 0.f : __expf(m_run - m_new);
+        float psum = 0.f;
+        uint32_t pa[2][2];  // the probabilities as row operand: [16-token step][tokens 2t.. | 2t+8..]
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            const float p0 = __expf(sc[nt][0] - m_new), p1 = __expf(sc[nt][1] - m_new);
+            psum += p0 + p1;
+            pa[nt >> 1][nt & 1] = pack2_bf16(p0, p1);
+        }
+        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+        l_run = l_run * corr + psum;
+        m_run = m_new;
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+            o[n][0] *= corr;
+            o[n][1] *= corr;
+        }
+        // weighted values: two 16-token steps x eight 8-channel blocks (two blocks per transposing matrix load)
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk) {
+            const int r = 16 * kk + 8 * ((lane >> 3) & 1) + (lane & 7);
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t b[4];
+                ldmatrix_x4_trans(vb + r * 128 + (((2 * np + (lane >> 4)) ^ (r & 7)) << 4), b);
+                mma_q8(o[2 * np], pa[kk][0], pa[kk][1], b[0], b[1]);
+                mma_q8(o[2 * np + 1], pa[kk][0], pa[kk][1], b[2], b[3]);
+            }
+        }
+        __syncwarp();  // every lane is done reading this step's buffers before the step after next refills them
+    }
+    if (g < group) {
+        float *part = a.partials + (((int64_t)si * a.max_chunks + tile) * a.hq + h * group + g) * (64 + 2);
+        if (t == 0) {
+            part[0] = m_run;
+            part[1] = l_run;
+        }
+#pragma unroll
+        for (int n = 0; n < 8; ++n) *reinterpret_cast<float2 *>(part + 2 + 8 * n + 2 * t) = make_float2(o[n][0], o[n][1]);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtype, int grid_chunks, cudaStream_t st) {
     dim3 grid(grid_chunks, (a.hkv + RW - 1) / RW, seqs.n);
+    if (dtype == KVCAR_BF16 && a.hq / a.hkv > 2) {
+        static bool configured = false;
+        if (!configured) {
+            cudaError_t e = cudaFuncSetAttribute(decode_raw_gq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GQ_SMEM);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        decode_raw_gq_kernel<<<grid, RW * 32, GQ_SMEM, st>>>(a, seqs);
+        return cudaGetLastError();
+    }
     if (dtype == KVCAR_F32)
         decode_raw_kernel<float><<<grid, RW * 32, 0, st>>>(a, seqs);
     else

@@ -149,6 +149,23 @@ def test_uncompressed_twin_and_mixed_stack(kernel):
         assert p.s.ctx.cache_bytes_per_token() == p.o.cache_bytes_per_token()
 
 
+@pytest.mark.parametrize("heads", [(32, 4), (12, 4), (6, 2)], ids=["group8", "group3", "group3_two_kv_heads"])
+def test_uncompressed_twin_with_query_groups(heads):
+    """Raw K/V pages with several query heads per KV head: the streaming kernel runs the group's dots on the
+    warp-level tensor op (groups of more than two heads).  Ragged tiles: a 32-token step that ends inside a tile,
+    a tile of one token, page boundaries inside a step; reuse redirects heads to the lower layer's rows."""
+    hq, hkv = heads
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, n_q_heads=hq, n_kv_heads=hkv, batch=4, reuse_frac=0.4)
+    p = Pair(w, max_seqs=4, max_pages=24, max_pages_per_seq=8, compress=False)
+    seqs = [0, 1, 2, 3]
+    p.open(seqs)
+    for s_, n in zip(seqs, (300, 129, 33, 1)):
+        p.prefill([s_], n)
+    assert all(p.s.ctx.layer_kernel(l) == B.KERNEL_RAW for l in range(w.n_layers))
+    for step in range(2):
+        _check_step(p.decode_step(seqs, step), "bf16", f"raw group {hq // hkv} step {step}")
+
+
 @pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
 def test_physical_page_permutation_is_bit_invariant(kernel):
     """The same logical cache laid out on different physical pages must give
