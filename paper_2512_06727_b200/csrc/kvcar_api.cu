@@ -713,8 +713,8 @@ static kvcar_status enqueue_decode_tiles(kvcar_ctx *c, int32_t layer, const Deco
     return KVCAR_OK;
 }
 
-static kvcar_status enqueue_combine(kvcar_ctx *c, const DecodeArgs &a, const SeqList &sl, cudaStream_t st) {
-    cudaError_t e = launch_combine(a, sl, c->cfg.storage, st);
+static kvcar_status enqueue_combine(kvcar_ctx *c, const DecodeArgs &a, const SeqList &sl, int n_chunks, cudaStream_t st) {
+    cudaError_t e = launch_combine(a, sl, c->cfg.storage, n_chunks, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "combine launch");
     ++c->launches;
     return KVCAR_OK;
@@ -744,7 +744,7 @@ kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *
     const int n_chunks = prepare_decode(c, layer, seqs, n_seqs, q, out, flags, a, sl);
     s = enqueue_decode_tiles(c, layer, a, sl, n_chunks, st);
     if (s != KVCAR_OK) return s;
-    return enqueue_combine(c, a, sl, st);
+    return enqueue_combine(c, a, sl, n_chunks, st);
 }
 
 kvcar_status kvcar_step_layer(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *k,
@@ -789,7 +789,7 @@ kvcar_status kvcar_step_layer(kvcar_ctx *c, int32_t layer, const int32_t *seqs, 
         s = enqueue_decode_tiles(c, layer, a, sl, n_chunks, st);
         if (s != KVCAR_OK) return s;
     }
-    return enqueue_combine(c, a, sl, st);
+    return enqueue_combine(c, a, sl, n_chunks, st);
 }
 
 kvcar_status kvcar_step_layer_host(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs,
@@ -1014,7 +1014,7 @@ extern "C" kvcar_status kvcar_decode_attention_static(kvcar_ctx *c, int32_t laye
         if (e != cudaSuccess) return cuda_fail(c, e, "decode launch");
         ++c->launches;
     }
-    e = launch_combine(a, sl, g.storage, st);
+    e = launch_combine(a, sl, g.storage, n_chunks, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "combine launch");
     ++c->launches;
     return KVCAR_OK;

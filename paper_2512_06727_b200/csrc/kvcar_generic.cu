@@ -448,6 +448,73 @@ __global__ void __launch_bounds__(32 * CB_WARPS) combine_kernel(const __grid_con
     }
 }
 
+// The same merge with one warp per (sequence, query head), for sequences of few tiles: no block-wide steps, eight
+// rows of the grid per CTA.  grid = ceil(hq * n_seqs / CB_WARPS); block = 32 * CB_WARPS.
+template <typename T>
+__global__ void __launch_bounds__(32 * CB_WARPS) combine_warp_kernel(const __grid_constant__ DecodeArgs a,
+                                                                     const __grid_constant__ SeqList seqs) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int hd = a.hd, hq = a.hq;  // hd <= 128
+    const int item = blockIdx.x * CB_WARPS + warp;
+    if (item >= hq * seqs.n) return;
+    const int si = item / hq, qh = item % hq;
+    const int seq = seqs.id[si];
+    const int L = a.seq_len[seq];
+    const int n_chunks = (L + a.chunk_tokens - 1) / a.chunk_tokens;
+    const int64_t stride = (int64_t)hq * (hd + 2);
+    const float *base = a.partials + ((int64_t)si * a.max_chunks * hq + qh) * (hd + 2);
+    float M = -INFINITY;
+    for (int ch = lane; ch < n_chunks; ch += 32) M = fmaxf(M, base[ch * stride]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float S = 0.f;
+    for (int ch = lane; ch < n_chunks; ch += 32) {
+        const float m = base[ch * stride], s = base[ch * stride + 1];
+        S += (m == -INFINITY) ? 0.f : s * expf(m - M);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
+    float av[4] = {0.f, 0.f, 0.f, 0.f};  // channels lane, lane + 32, lane + 64, lane + 96
+#pragma unroll 4
+    for (int ch = 0; ch < n_chunks; ++ch) {
+        const float *part = base + ch * stride;
+        const float m = part[0];
+        const float w = (m == -INFINITY) ? 0.f : expf(m - M);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (lane + 32 * j < hd) av[j] = fmaf(w, part[2 + lane + 32 * j], av[j]);
+    }
+    float c0 = 1.f, c1 = 0.f;
+    const T *vc = nullptr;
+    if (a.flags & KVCAR_INCLUDE_CURRENT_EXACT) {
+        const int g = qh / (hq / a.hkv);
+        const int W = a.hkv * hd;
+        const T *kc = reinterpret_cast<const T *>(a.plan->cur[0][g]) + (int64_t)seq * W + a.plan->cur_head[0][g] * hd;
+        vc = reinterpret_cast<const T *>(a.plan->cur[1][g]) + (int64_t)seq * W + a.plan->cur_head[1][g] * hd;
+        const T *qg = reinterpret_cast<const T *>(a.q) + ((int64_t)si * hq + qh) * hd;
+        float prod = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (lane + 32 * j < hd) prod = fmaf(ld(qg + lane + 32 * j), ld(kc + lane + 32 * j), prod);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) prod += __shfl_xor_sync(0xffffffffu, prod, o);
+        const float sc = prod * a.scale;
+        const float Mn = fmaxf(M, sc);
+        c0 = (M == -INFINITY) ? 0.f : expf(M - Mn);
+        c1 = expf(sc - Mn);
+        S = S * c0 + c1;
+    }
+    T *o = reinterpret_cast<T *>(a.out) + ((int64_t)si * hq + qh) * hd;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int c = lane + 32 * j;
+        if (c < hd) {
+            const float acc = av[j] * c0 + (vc ? ld(vc + c) * c1 : 0.f);
+            st(o + c, S > 0.f ? acc / S : 0.f);
+        }
+    }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------
@@ -497,7 +564,18 @@ cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int 
     return cudaGetLastError();
 }
 
-cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, cudaStream_t st) {
+cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, int n_chunks, cudaStream_t st) {
+    // Many (sequence, query head) rows of few tiles each: one warp per row.  Otherwise a CTA per row, which merges
+    // a row's tiles in parallel (measured: 1024 rows x 16 tiles are 2 us per call faster with warps; 96 rows x
+    // 8 tiles and 384 rows x 33 tiles are faster with CTAs).
+    if (n_chunks <= 32 && a.hq * seqs.n >= 512) {
+        const int grid = (a.hq * seqs.n + CB_WARPS - 1) / CB_WARPS;
+        if (dtype == KVCAR_F32)
+            combine_warp_kernel<float><<<grid, 32 * CB_WARPS, 0, st>>>(a, seqs);
+        else
+            combine_warp_kernel<__nv_bfloat16><<<grid, 32 * CB_WARPS, 0, st>>>(a, seqs);
+        return cudaGetLastError();
+    }
     dim3 grid(a.hq, seqs.n);
     if (dtype == KVCAR_F32)
         combine_kernel<float><<<grid, 32 * CB_WARPS, 0, st>>>(a, seqs);

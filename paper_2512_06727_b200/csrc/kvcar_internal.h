@@ -110,7 +110,8 @@ cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int 
                                   int grid_chunks, cudaStream_t st);
 // raw K/V layers (no autoencoder), head_dim 64, <= 8 query heads per KV head (kvcar_raw.cu)
 cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtype, int grid_chunks, cudaStream_t st);
-cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, cudaStream_t st);
+// n_chunks: tiles of the longest listed sequence (picks the kernel: a warp or a CTA per sequence and query head)
+cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, int n_chunks, cudaStream_t st);
 size_t decode_generic_smem(int hq, int hd, int max_d, int max_m);
 
 }  // namespace kvcar

@@ -204,7 +204,8 @@ __global__ void __launch_bounds__(RW * 32, 4) decode_raw_kernel(const __grid_con
 constexpr int GQ_STEP = 32;                      // tokens per step
 constexpr int GQ_BUF = GQ_STEP * 64 * 2;         // bytes of one K (or V) step buffer: 32 rows x 128 B
 constexpr int GQ_WARP_SMEM = 4 * GQ_BUF;         // K and V, two steps each
-constexpr int GQ_SMEM = RW * GQ_WARP_SMEM;
+constexpr int GQ_RW = 2;                         // warps (= KV heads) per CTA: small CTAs pack the SMs evenly
+constexpr int GQ_SMEM = GQ_RW * GQ_WARP_SMEM;
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
@@ -234,11 +235,11 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
-__global__ void __launch_bounds__(RW * 32) decode_raw_gq_kernel(const __grid_constant__ DecodeArgs a,
+__global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_constant__ DecodeArgs a,
                                                                const __grid_constant__ SeqList seqs) {
     extern __shared__ __align__(128) uint8_t gq_smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x, h = blockIdx.y * RW + warp, si = blockIdx.z;
+    const int tile = blockIdx.x, h = blockIdx.y * GQ_RW + warp, si = blockIdx.z;
     if (h >= a.hkv) return;
     const int seq = seqs.id[si];
     const int L = a.seq_len[seq];
@@ -377,7 +378,8 @@ cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtyp
             if (e != cudaSuccess) return e;
             configured = true;
         }
-        decode_raw_gq_kernel<<<grid, RW * 32, GQ_SMEM, st>>>(a, seqs);
+        grid.y = (a.hkv + GQ_RW - 1) / GQ_RW;
+        decode_raw_gq_kernel<<<grid, GQ_RW * 32, GQ_SMEM, st>>>(a, seqs);
         return cudaGetLastError();
     }
     if (dtype == KVCAR_F32)

@@ -229,6 +229,23 @@ def test_tensor_kernel_variants_walk_several_pairs(shape):
     _check_step(p.decode_step(seqs, 0), "bf16", shape)
 
 
+@pytest.mark.parametrize("storage", ["bf16", "f32"])
+def test_many_short_sequences_merge_one_warp_per_row(storage):
+    """512 (sequence, query head) rows of at most three tiles: the tile partials and the current token are merged
+    by the one-warp-per-row kernel (fewer rows or longer sequences take the CTA-per-row kernel of the other tests).
+    Lengths include 0 (current token only) and exact tile multiples."""
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=16, cached_tokens=0, decode_steps=1, reuse_frac=0.25,
+                     storage=storage)
+    p = Pair(w, max_seqs=16, max_pages=16 * 6, max_pages_per_seq=6)
+    seqs = list(range(16))
+    p.open(seqs)
+    for s_, n in zip(seqs, (0, 1, 127, 128, 129, 256, 300, 64, 5, 200, 257, 31, 33, 255, 90, 130)):
+        if n:
+            p.prefill([s_], n)
+    _check_step(p.decode_step(seqs, 0), storage, f"warp merge {storage}")
+    _check_step(p.decode_step(seqs, 1, include_current=False), storage, f"warp merge, cached only, {storage}")
+
+
 def test_fp32_stack_with_reuse_generic():
     """fp32 mode on a multi-layer stack with chains of reuse; 1e-4 absolute."""
     w = synth.scaled(synth.CONFIGS["c2"], n_layers=4, batch=2, storage="f32", reuse_frac=0.5)
