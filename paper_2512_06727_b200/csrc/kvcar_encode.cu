@@ -167,16 +167,16 @@ __global__ void __launch_bounds__(NW * 32)
                     reinterpret_cast<const uint4 *>(src + (int64_t)r * a.kv_width)[cv];
             }
         }
-        if (!compressed) {  // raw layer: copy the stored heads' slices into the cache rows
-            if (blockIdx.x == 0) {
-                T *pool = reinterpret_cast<T *>(pl.pool);
-                for (int idx = threadIdx.x; idx < rows_here * in_dim; idx += blockDim.x) {
-                    const int rr = idx / in_dim, c = idx % in_dim, r = r0 + rr;
-                    const int seq = seqs.id[r], t = a.seq_len[seq];
-                    const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
-                    const int64_t pr = (int64_t)page * a.page_tokens + t % a.page_tokens;
-                    pool[pr * pl.width + c] = src[(int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd];
-                }
+        if (!compressed) {  // raw layer: copy the stored heads' slices into the cache rows, 16 bytes at a time
+            T *pool = reinterpret_cast<T *>(pl.pool);
+            const int nv = in_dim / VL;
+            for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < rows_here * nv; idx += gridDim.x * blockDim.x) {
+                const int rr = idx / nv, c = (idx % nv) * VL, r = r0 + rr;
+                const int seq = seqs.id[r], t = a.seq_len[seq];
+                const int page = a.block_table[(int64_t)seq * a.max_pages_per_seq + t / a.page_tokens];
+                const int64_t pr = (int64_t)page * a.page_tokens + t % a.page_tokens;
+                *reinterpret_cast<uint4 *>(pool + pr * pl.width + c) =
+                    Vec16<T>::load(src + (int64_t)r * a.kv_width + pl.heads[c / a.hd] * a.hd + c % a.hd);
             }
             return;
         }
