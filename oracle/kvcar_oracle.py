@@ -89,6 +89,45 @@ def int8_dequantize(q: np.ndarray, scale: float, zeropoint: float) -> np.ndarray
 
 
 # --------------------------------------------------------------------------
+# Alg. 2, first steps: which heads may reuse the layer below
+# --------------------------------------------------------------------------
+def head_l1_distance(x: np.ndarray, n_kv_heads: int) -> np.ndarray:
+    """Alg. 2 ("inter layer L1 norm between heads of adjacent layers"; Sec. "Network
+    Architecture": the L1 norm "captures the absolute differences between their key
+    and value matrices").  x: recorded K (or V) rows, [n_layers][n_rows][n_kv_heads *
+    head_dim].  Returns D [n_layers - 1][n_kv_heads]: D[l-1][h] = mean over the rows and
+    over head h's channels of |x[l] - x[l-1]|, i.e. the L1 norm of the difference of
+    head h's matrix in layers l and l-1 divided by its element count (the paper does
+    not say whether it normalises; dividing makes mini-batches of different sizes
+    average as the text says they are averaged).  Same head index in both layers."""
+    x = np.asarray(x, dtype=np.float64)
+    n_layers, n_rows, width = x.shape
+    hd = width // n_kv_heads
+    out = np.zeros((n_layers - 1, n_kv_heads))
+    for l in range(1, n_layers):
+        diff = np.abs(x[l] - x[l - 1])
+        for h in range(n_kv_heads):
+            out[l - 1, h] = diff[:, h * hd:(h + 1) * hd].sum() / (n_rows * hd)
+    return out
+
+
+def reuse_map_from_l1(dist: np.ndarray, n_reuse: int) -> np.ndarray:
+    """Alg. 2, next step: the heads with the smallest distance to the layer below
+    reuse it ("a threshold is empirically determined": here the threshold is given as
+    a count, the n_reuse closest heads; equal distances go to the lower layer, then
+    the lower head).  dist: [n_layers - 1][n_kv_heads] as returned above.  Returns the
+    table in the form the cache takes it: int32 [n_layers * n_kv_heads], -1 = own
+    data, else the head index in layer l-1 (always the same index here)."""
+    dist = np.asarray(dist, dtype=np.float64)
+    n_pairs, n_kv_heads = dist.shape
+    order = sorted(range(n_pairs * n_kv_heads), key=lambda i: (dist[i // n_kv_heads, i % n_kv_heads], i))
+    src = np.full((n_pairs + 1) * n_kv_heads, -1, dtype=np.int32)
+    for i in order[:n_reuse]:
+        src[n_kv_heads + i] = i % n_kv_heads
+    return src
+
+
+# --------------------------------------------------------------------------
 # the autoencoder halves
 # --------------------------------------------------------------------------
 def mlp_forward(x: np.ndarray, w1, b1, bn, w2, b2, leaky_slope: float, bn_eps: float) -> np.ndarray:

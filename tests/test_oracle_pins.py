@@ -536,3 +536,65 @@ def test_reuse_map_generator_counts():
         assert np.all(src[:w.n_kv_heads] == -1)
         again = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
         assert np.array_equal(src, again)
+
+
+# ---------------------------------------------------------------- Alg. 2: head distances and the reuse choice
+def test_head_l1_distance_closed_forms_and_brute_force():
+    """Alg. 2, "inter layer L1 norm between heads of adjacent layers", pinned by cases with a known answer:
+    equal layers -> 0; a per-head constant offset -> its magnitude; loops written out on a tiny case (which
+    catches a wrong layer pairing, a wrong head slice or a wrong divisor); scaling; row order."""
+    rng = np.random.default_rng(5)
+    L, R, H, hd = 4, 7, 3, 4
+    base = rng.normal(size=(R, H * hd))
+    # (1) identical layers
+    x = np.stack([base] * L)
+    assert np.array_equal(orc.head_l1_distance(x, H), np.zeros((L - 1, H)))
+    # (2) layer l = layer l-1 + delta[l][h] on every channel of head h: distance = |delta|
+    delta = rng.normal(size=(L, H))
+    x = np.zeros((L, R, H * hd))
+    x[0] = base
+    for l in range(1, L):
+        x[l] = x[l - 1] + np.repeat(delta[l], hd)[None, :]
+    np.testing.assert_allclose(orc.head_l1_distance(x, H), np.abs(delta[1:]), rtol=0, atol=1e-12)
+    # (3) brute force, every index written out
+    x = rng.normal(size=(L, R, H * hd))
+    want = np.zeros((L - 1, H))
+    for l in range(1, L):
+        for h in range(H):
+            tot = 0.0
+            for r in range(R):
+                for c in range(hd):
+                    tot += abs(x[l][r][h * hd + c] - x[l - 1][r][h * hd + c])
+            want[l - 1][h] = tot / (R * hd)
+    got = orc.head_l1_distance(x, H)
+    np.testing.assert_allclose(got, want, rtol=1e-13, atol=0)
+    assert not np.allclose(got, orc.head_l1_distance(x[::-1], H)[::-1][:, ::-1])    # heads are not interchangeable
+    # (4) |a| D(x) = D(a x); the order of the rows is irrelevant; a constant added to every layer cancels
+    np.testing.assert_allclose(orc.head_l1_distance(-2.5 * x, H), 2.5 * got, rtol=1e-13)
+    np.testing.assert_allclose(orc.head_l1_distance(x[:, rng.permutation(R)], H), got, rtol=1e-13)
+    np.testing.assert_allclose(orc.head_l1_distance(x + 3.0, H), got, rtol=1e-12)
+    # (5) mini-batches of equal size average to the distance of their union (the text averages over mini-batches)
+    a, b = rng.normal(size=(L, R, H * hd)), rng.normal(size=(L, R, H * hd))
+    both = np.concatenate([a, b], axis=1)
+    np.testing.assert_allclose(0.5 * (orc.head_l1_distance(a, H) + orc.head_l1_distance(b, H)),
+                               orc.head_l1_distance(both, H), rtol=1e-13)
+
+
+def test_reuse_map_from_l1_picks_the_closest_heads():
+    """Alg. 2: heads whose distance to the layer below is smallest reuse it.  Hand-made distances with a known
+    ranking (including a tie) and the table format the cache expects (layer 0 never reuses; entry = same head)."""
+    dist = np.array([[0.9, 0.1, 0.5],       # layer 1 vs 0
+                     [0.1, 0.7, 0.3],       # layer 2 vs 1   (0.1 ties with layer 1, head 1: the lower layer wins)
+                     [0.2, 0.8, 0.6]])      # layer 3 vs 2
+    none = orc.reuse_map_from_l1(dist, 0)
+    assert none.dtype == np.int32 and none.tolist() == [-1] * 12
+    one = orc.reuse_map_from_l1(dist, 1)
+    assert one.tolist() == [-1, -1, -1, -1, 1, -1, -1, -1, -1, -1, -1, -1]
+    four = orc.reuse_map_from_l1(dist, 4)
+    # ranking: (1,1)=0.1, (2,0)=0.1, (3,0)=0.2, (2,2)=0.3
+    assert four.tolist() == [-1, -1, -1, -1, 1, -1, 0, -1, 2, 0, -1, -1]
+    assert orc.reuse_map_from_l1(dist, 9).tolist() == [-1, -1, -1, 0, 1, 2, 0, 1, 2, 0, 1, 2]
+    # the table is accepted by the cache model and resolves through chains (layer 3 head 0 -> layer 1 head 0)
+    o = KVCAROracle(4, 3, 3, 4, page_tokens=2, max_seqs=1, max_pages=4, storage="exact")
+    o.set_reuse_map(four, four)
+    assert o.resolve(3, 0, K)[:2] == (1, 0)
