@@ -51,6 +51,9 @@ def parse():
     ap.add_argument("--api", default="fused", choices=["fused", "split"],
                     help="a layer's step through kvcar_step_layer (one call; the tile kernel runs beside the encoder) "
                          "or through kvcar_encode_append + kvcar_decode_attention")
+    ap.add_argument("--head-l1", action="store_true",
+                    help="instead of the decode step: time Alg. 2's head-distance reduction on K rows shaped like "
+                         "the workload (layers x batch*cached_tokens x KV width) and print its own JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle sample")
@@ -340,10 +343,63 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------
+def run_head_l1(args):
+    """Alg. 2's statistic as a streaming reduction: GB/s of activations read against the measured copy bandwidth."""
+    import torch
+    from oracle import kvcar_oracle as orc
+    from paper_2512_06727_b200 import binding as B
+    w = workload_of(args)
+    n_rows = w.batch * w.cached_tokens
+    hkv, hd, L = w.n_kv_heads, w.head_dim, w.n_layers
+    g = torch.Generator(device="cuda").manual_seed(w.seed)
+    x = torch.empty(L, n_rows, hkv * hd, dtype=torch.bfloat16, device="cuda")
+    x[0] = torch.randn(n_rows, hkv * hd, generator=g, device="cuda")
+    for l in range(1, L):
+        x[l] = x[l - 1].float() + 0.3 * torch.randn(n_rows, hkv * hd, generator=g, device="cuda")
+    nbytes = B.head_l1_scratch_bytes(L, hkv, n_rows)
+    scratch = torch.empty(nbytes // 4 + 4, device="cuda")
+    dist_ = torch.empty(L - 1, hkv, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    K_, W_ = args.steps, max(args.warmup, 3)
+    ev = []
+    for i in range(W_ + K_):
+        flush.fill_(i & 0xFF)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        B.head_l1_distance(L, hkv, hd, B.BF16, x.data_ptr(), n_rows, scratch.data_ptr(), nbytes, dist_.data_ptr(), stream)
+        b.record()
+        if i >= W_:
+            ev.append((a, b))
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in ev) / len(ev)
+    byts = float(x.numel() * 2)
+    peaks = measured_peaks()
+    gbs = byts / (ms / 1e3) / 1e9
+    # parity on a sample of rows the oracle does in a moment (the rows' share of every sum is the same reduction)
+    rows = min(n_rows, 256)
+    sub = x[:, :rows].contiguous()
+    B.head_l1_distance(L, hkv, hd, B.BF16, sub.data_ptr(), rows, scratch.data_ptr(), nbytes, dist_.data_ptr(), stream)
+    torch.cuda.synchronize()
+    want = orc.head_l1_distance(sub.float().cpu().numpy().astype("float64"), hkv)
+    err = float(abs(dist_.cpu().numpy() - want).max() / want.max())
+    print(json.dumps({"metric": "head L1 distance (Alg. 2) activations read", "value": gbs, "unit": "GB/s", "n_gpus": 1,
+                      "steps": K_, "warmup": W_, "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16",
+                      "data": "synthetic", "config": {"workload": w.name + "_head_l1", "layers": L, "rows": n_rows,
+                                                       "kv_width": hkv * hd, "l2": "flushed between launches"},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                                   "algorithmic_bytes_per_launch": byts},
+                      "max_rel_err_vs_oracle_on_256_rows": err, "gpu_launches": 2 * K_}))
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.head_l1:
+        run_head_l1(args)
         return
     import torch
     import torch.distributed as dist

@@ -287,6 +287,42 @@ kvcar_status kvcar_layer_kernel(kvcar_ctx *ctx, int32_t layer, int32_t *kernel);
 kvcar_status kvcar_sync_status(kvcar_ctx *ctx, void *stream);
 const char *kvcar_last_error(kvcar_ctx *ctx);
 
+/* ---- choosing the reuse map (Alg. 2, its first three steps) -------------------
+ *
+ * These calls need no context: they work on activations recorded by the caller.
+ *
+ * kvcar_head_l1_distance: "Calculate inter layer L1 norm between heads of
+ * adjacent layers" (Alg. 2; Sec. "Network Architecture": the norm "captures the
+ * absolute differences between their key and value matrices").
+ * x: DEVICE [n_layers][n_rows][n_kv_heads * head_dim], storage type `storage`
+ * (KVCAR_F32 / KVCAR_BF16), 16-byte aligned: the K (or the V) rows of one
+ * mini-batch, n_rows = sequences x tokens.  dist: DEVICE float
+ * [n_layers - 1][n_kv_heads]; dist[l-1][h] = mean over rows and over head h's
+ * head_dim channels of |x[l] - x[l-1]| (the paper does not say whether the norm
+ * is normalised; dividing by the element count lets mini-batches of different
+ * sizes be averaged, as the text averages them - that average is the caller's).
+ * scratch: DEVICE, at least kvcar_head_l1_scratch_bytes() bytes, 16-byte
+ * aligned, contents irrelevant before and after.  Sums are taken in a fixed
+ * order: the result is the same on every run.  head_dim * element size must be
+ * a multiple of 16 bytes.  Errors: KVCAR_ERR_INVALID_ARG (pointers, alignment,
+ * sizes), KVCAR_ERR_WORKSPACE (scratch too small), KVCAR_ERR_CUDA (launch).
+ * Returns after enqueuing on `stream`.
+ */
+kvcar_status kvcar_head_l1_scratch_bytes(int32_t n_layers, int32_t n_kv_heads, int64_t n_rows, size_t *bytes);
+kvcar_status kvcar_head_l1_distance(int32_t n_layers, int32_t n_kv_heads, int32_t head_dim, int32_t storage, const void *x,
+                                    int64_t n_rows, void *scratch, size_t scratch_bytes, float *dist, void *stream);
+/*
+ * "Based on L1 norm, the key and value heads in the particular layers are
+ * reused by the key and value in the previous layer" (Alg. 2): the n_reuse heads
+ * with the smallest distance reuse the same head of the layer below (the
+ * paper's empirical threshold, given as a count; equal distances: lower layer,
+ * then lower head, first).  dist: HOST float [n_layers - 1][n_kv_heads] (no NaN);
+ * src: HOST int32 [n_layers * n_kv_heads], written in the form
+ * kvcar_set_reuse_map takes (-1 = own data).  Host only, no GPU needed.
+ */
+kvcar_status kvcar_reuse_map_from_l1(const float *dist, int32_t n_layers, int32_t n_kv_heads, int32_t n_reuse,
+                                     int32_t *src);
+
 #ifdef __cplusplus
 }
 #endif

@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
-from typing import Optional, Sequence, Tuple
+from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
@@ -31,6 +31,7 @@ EXPORTS = [
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
     "kvcar_last_error",
+    "kvcar_head_l1_scratch_bytes", "kvcar_head_l1_distance", "kvcar_reuse_map_from_l1",
 ]
 
 
@@ -59,7 +60,18 @@ def lib_path() -> str:
     return _build.LIB
 
 
+_LIB: Optional[C.CDLL] = None
+
+
 def load() -> C.CDLL:
+    """The library, built if its sources are newer, loaded once per process."""
+    global _LIB
+    if _LIB is None:
+        _LIB = _load()
+    return _LIB
+
+
+def _load() -> C.CDLL:
     path = lib_path()
     if _build.needs_build():
         _build.build()
@@ -94,6 +106,9 @@ def load() -> C.CDLL:
         "kvcar_launch_count": [vp, C.POINTER(C.c_int64)],
         "kvcar_layer_kernel": [vp, i32, ip],
         "kvcar_sync_status": [vp, vp],
+        "kvcar_head_l1_scratch_bytes": [i32, i32, C.c_int64, C.POINTER(sz)],
+        "kvcar_head_l1_distance": [i32, i32, i32, i32, vp, C.c_int64, vp, sz, vp, vp],
+        "kvcar_reuse_map_from_l1": [C.POINTER(C.c_float), i32, i32, i32, ip],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -102,6 +117,33 @@ def load() -> C.CDLL:
     lib.kvcar_last_error.argtypes = [vp]
     lib.kvcar_last_error.restype = C.c_char_p
     return lib
+
+
+# -- the context-free calls: choosing the reuse map (argument marshalling only) -------------------
+def head_l1_scratch_bytes(n_layers: int, n_kv_heads: int, n_rows: int) -> int:
+    out = C.c_size_t()
+    st = load().kvcar_head_l1_scratch_bytes(n_layers, n_kv_heads, n_rows, C.byref(out))
+    if st != 0:
+        raise KvcarError(st, "kvcar_head_l1_scratch_bytes")
+    return out.value
+
+
+def head_l1_distance(n_layers: int, n_kv_heads: int, head_dim: int, storage: int, x: int, n_rows: int, scratch: int,
+                     scratch_bytes: int, dist: int, stream: int = 0) -> None:
+    """x, scratch, dist: device addresses (see kvcar_head_l1_distance in kvcar.h)."""
+    st = load().kvcar_head_l1_distance(n_layers, n_kv_heads, head_dim, storage, x, n_rows, scratch, scratch_bytes, dist,
+                                       stream)
+    if st != 0:
+        raise KvcarError(st, "kvcar_head_l1_distance")
+
+
+def reuse_map_from_l1(dist: Sequence[float], n_layers: int, n_kv_heads: int, n_reuse: int) -> List[int]:
+    arr = (C.c_float * len(dist))(*dist)
+    src = (C.c_int32 * (n_layers * n_kv_heads))()
+    st = load().kvcar_reuse_map_from_l1(arr, n_layers, n_kv_heads, n_reuse, src)
+    if st != 0:
+        raise KvcarError(st, "kvcar_reuse_map_from_l1")
+    return list(src)
 
 
 def _ints(seq: Sequence[int]):

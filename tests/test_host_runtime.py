@@ -165,3 +165,30 @@ def test_launching_calls_need_bound_memory():
     assert e.value.status == 2
     with pytest.raises(B.KvcarError):
         B.Context(1, 5, 2, 64, 64, 2, 4, 2, B.BF16)      # query heads not a multiple of KV heads
+
+
+def test_reuse_map_from_l1_matches_oracle_bit_for_bit():
+    """Alg. 2's choice of reused heads is integer work on the host: the library's table equals the oracle's for
+    random distances (with planted ties) at every count, and bad arguments are refused."""
+    from oracle import kvcar_oracle as orc
+    rng = np.random.default_rng(11)
+    for (L, H) in ((12, 12), (22, 4), (2, 1)):
+        dist = rng.random((L - 1, H)).astype(np.float32)
+        if dist.size > 3:
+            dist.flat[3] = dist.flat[0]          # ties: the lower (layer, head) goes first
+            dist.flat[-1] = dist.flat[0]
+        for n_reuse in sorted({0, 1, dist.size // 4, dist.size}):
+            got = B.reuse_map_from_l1(dist.ravel().tolist(), L, H, n_reuse)
+            want = orc.reuse_map_from_l1(dist.astype(np.float64), n_reuse)
+            assert got == want.tolist(), (L, H, n_reuse)
+            assert sum(1 for v in got if v >= 0) == n_reuse and all(v == -1 for v in got[:H])
+    with pytest.raises(B.KvcarError):
+        B.reuse_map_from_l1([0.1, 0.2], 2, 2, 3)              # more heads than there are
+    with pytest.raises(B.KvcarError):
+        B.reuse_map_from_l1([0.1, float("nan")], 2, 2, 1)
+    # size query and argument checks of the distance call need no GPU
+    assert B.head_l1_scratch_bytes(12, 12, 8192) == (8192 // 8) * 11 * 12 * 4
+    with pytest.raises(B.KvcarError):
+        B.head_l1_scratch_bytes(1, 12, 8192)                  # one layer has no layer below
+    with pytest.raises(B.KvcarError):
+        B.head_l1_distance(12, 12, 60, B.BF16, 16, 8, 16, 1 << 20, 16)   # a 60-wide head is not whole 16-byte chunks
