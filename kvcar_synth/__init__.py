@@ -74,7 +74,7 @@ def normal(shape, seed: int, *stream, storage: str = "f32", scale: float = 1.0) 
 
 
 # --------------------------------------------------------------------------
-# workload descriptions (BASELINE configs)
+# workload descriptions (the benchmark configurations)
 # --------------------------------------------------------------------------
 @dataclass(frozen=True)
 class Workload:

@@ -26,7 +26,7 @@ def _check_step(res, storage, what):
 
 
 def test_config1_fp32_single_layer():
-    """BASELINE config 1 exactly: one GPT-2-small-shaped layer, 768->384, batch 1,
+    """Configuration 1 exactly: one GPT-2-small-shaped layer, 768->384, batch 1,
     128 cached tokens, one decode step, fp32, no reuse; max abs error <= 1e-4."""
     w = synth.CONFIGS["c1"]
     p = Pair(w, max_seqs=1, max_pages=4, max_pages_per_seq=4)
