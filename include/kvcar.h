@@ -273,9 +273,10 @@ kvcar_status kvcar_pool_layout(kvcar_ctx *ctx, int32_t layer, int32_t which, siz
  * neither autoencoders nor reuse (Eq. 3 per token and sequence). */
 kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *ctx, double *compressed, double *uncompressed);
 /* Algorithmic work of one kvcar_decode_attention call on `layer` per cached
- * token: latent bytes read and floating-point operations (decoder + attention),
- * following the reuse map (each distinct source layer is read and passed
- * through its first decoder layer once). */
+ * token: cache bytes read and floating-point operations (decoder + attention),
+ * following the reuse map (each distinct source layer's latent row is read whole
+ * and passed through its first decoder layer once; of a raw row only the needed
+ * heads' slices are read). */
 kvcar_status kvcar_layer_work_per_token(kvcar_ctx *ctx, int32_t layer, double *bytes, double *flops);
 /* Number of kernels the library has launched so far on this context. */
 kvcar_status kvcar_launch_count(kvcar_ctx *ctx, int64_t *count);

@@ -880,7 +880,8 @@ kvcar_status kvcar_layer_work_per_token(kvcar_ctx *c, int32_t layer, double *byt
         for (int s = 0; s < c->cfg.n_layers; ++s) {
             if (!need[s]) continue;
             const AEHost &a = c->ae[s * 2 + which];
-            b += (double)stored_width(c, s, which) * c->elem;
+            // a latent row mixes all heads of its layer and is read whole; of a raw row only the needed heads' slices
+            b += a.set ? (double)stored_width(c, s, which) * c->elem : (double)need[s] * hd * c->elem;
             if (a.set) f += 2.0 * a.latent * a.hidden + 2.0 * a.hidden * hd * need[s];
         }
     }

@@ -1,13 +1,17 @@
 // Decode attention over layers that store raw K/V rows (no autoencoder): the uncompressed twin of the latent
-// path.  There is no decoder, so the cost is reading every cached K and V row once: the kernel is built to keep
-// HBM busy, not the tensor cores.
+// path.  There is no decoder, so the cost is reading every cached K and V row once: the kernels are built to keep
+// HBM busy.  One warp owns one (sequence, 128-token tile, KV head); the tile's (max, sum, weighted values) go to
+// the split-KV partials; the combine kernel merges tiles and the exact current token.  A reused head reads the
+// lower layer's rows.
 //
-// One warp owns one (sequence, 128-token tile, KV head).  K phase: lane = token; the lane reads its token's
-// 64-wide K slice (128 B in 16-byte loads) and dots it with the group's pre-scaled queries (shared memory,
-// broadcast reads).  Online softmax over the tile's four 32-token groups (shuffle max / sum).  V phase: lane =
-// channel pair; the warp reads one V row per step (128 contiguous bytes), the row index and the probabilities
-// come from the owning lane by shuffle.  The tile's (max, sum, weighted values) go to the split-KV partials;
-// the combine kernel merges tiles and the exact current token.  A reused head reads the lower layer's rows.
+// bf16 rows (decode_raw_gq_kernel, below): 32 tokens at a time through shared memory into the warp-level tensor
+// op, for every group size (a group of one query head is padded like any other; the products are nowhere near
+// the limit).
+//
+// fp32 rows (decode_raw_kernel): K phase with lane = token; the lane reads its token's 64-wide K slice in 16-byte
+// loads and dots it with the group's pre-scaled queries (shared memory, broadcast reads).  Online softmax over
+// the tile's four 32-token groups (shuffle max / sum).  V phase: lane = channel pair; the warp reads one V row
+// per step, the row index and the probabilities come from the owning lane through shared memory.
 #include "kvcar_internal.h"
 
 namespace kvcar {
@@ -194,13 +198,15 @@ __global__ void __launch_bounds__(RW * 32, 4) decode_raw_kernel(const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Query groups of more than two heads, bf16 rows: the dots of a group against a row are a small matrix product,
-// and on the CUDA cores they, not HBM, set the pace (8 heads: 1024 FMA per cached row and KV head).  Same
+// bf16 rows.  With several query heads per KV head the dots of a group against a row are a small matrix product,
+// and on the CUDA cores they, not HBM, set the pace (8 heads: 1024 FMA per cached row and KV head); and even with
+// one head per group a warp that walks its tile with plain loads keeps too few bytes in flight.  Same
 // decomposition (one warp per sequence, 128-token tile and KV head), but 32 tokens at a time go through shared
 // memory (cp.async, 16-byte chunks swizzled by row, the next 32 tokens in flight meanwhile) into the warp-level
 // tensor op: scores^T[8 queries x 8 tokens] = Q . K^T with the K rows as the "column-major" operand they already
 // are; the probabilities come out in the layout the next product wants as its row operand (queries x tokens), and
-// V enters through transposing matrix loads.  Online softmax across the four 32-token steps, fp32.
+// V enters through transposing matrix loads.  Online softmax across the four 32-token steps, fp32.  Groups of
+// fewer than 8 heads leave the other operand rows zero.
 constexpr int GQ_STEP = 32;                      // tokens per step
 constexpr int GQ_BUF = GQ_STEP * 64 * 2;         // bytes of one K (or V) step buffer: 32 rows x 128 B
 constexpr int GQ_WARP_SMEM = 4 * GQ_BUF;         // K and V, two steps each
@@ -371,12 +377,14 @@ __global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_
 
 cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtype, int grid_chunks, cudaStream_t st) {
     dim3 grid(grid_chunks, (a.hkv + RW - 1) / RW, seqs.n);
-    if (dtype == KVCAR_BF16 && a.hq / a.hkv > 2) {
-        static bool configured = false;
-        if (!configured) {
+    if (dtype == KVCAR_BF16) {
+        static bool configured[64] = {};  // per device: the attribute belongs to the device's copy of the kernel
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev < 0 || dev >= 64 || !configured[dev]) {
             cudaError_t e = cudaFuncSetAttribute(decode_raw_gq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GQ_SMEM);
             if (e != cudaSuccess) return e;
-            configured = true;
+            if (dev >= 0 && dev < 64) configured[dev] = true;
         }
         grid.y = (a.hkv + GQ_RW - 1) / GQ_RW;
         decode_raw_gq_kernel<<<grid, GQ_RW * 32, GQ_SMEM, st>>>(a, seqs);

@@ -1502,12 +1502,15 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     using Kernel = void (*)(const DecodeArgs, const SeqList, const TileIndex, const PairLaunch);
     static const Kernel kernels[4] = {decode_pair_kernel<false, false>, decode_pair_kernel<false, true>,
                                       decode_pair_kernel<true, false>, decode_pair_kernel<true, true>};
-    static int configured_smem[4] = {0, 0, 0, 0};
+    static int configured_smem[64][4] = {};  // per device: the attribute belongs to the device's copy of the kernel
     const int ki = (lay.group_mma ? 2 : 0) + (lc.max_m <= 256 ? 1 : 0);
-    if (smem > configured_smem[ki]) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const bool known = dev >= 0 && dev < 64;
+    if (!known || smem > configured_smem[dev][ki]) {
         cudaError_t e = cudaFuncSetAttribute(kernels[ki], cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        configured_smem[ki] = smem;
+        if (known) configured_smem[dev][ki] = smem;
     }
     kernels[ki]<<<grid, NTHREADS, smem, st>>>(a, seqs, tix, lay);
     return cudaGetLastError();
