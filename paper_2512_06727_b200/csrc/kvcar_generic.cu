@@ -448,8 +448,10 @@ __global__ void __launch_bounds__(32 * CB_WARPS) combine_kernel(const __grid_con
     }
 }
 
-// The same merge with one warp per (sequence, query head), for sequences of few tiles: no block-wide steps, eight
-// rows of the grid per CTA.  grid = ceil(hq * n_seqs / CB_WARPS); block = 32 * CB_WARPS.
+// The same merge with one warp per (sequence, query head), for sequences of at most 32 tiles: lane c owns tile c's
+// (maximum, sum); the weighted values of all tiles are fetched in one batch of independent loads, and the current
+// token's operands are requested before anything else, so the whole merge is about two memory round trips.
+// grid = ceil(hq * n_seqs / CB_WARPS); block = 32 * CB_WARPS.
 template <typename T>
 __global__ void __launch_bounds__(32 * CB_WARPS) combine_warp_kernel(const __grid_constant__ DecodeArgs a,
                                                                      const __grid_constant__ SeqList seqs) {
@@ -459,43 +461,72 @@ __global__ void __launch_bounds__(32 * CB_WARPS) combine_warp_kernel(const __gri
     if (item >= hq * seqs.n) return;
     const int si = item / hq, qh = item % hq;
     const int seq = seqs.id[si];
-    const int L = a.seq_len[seq];
-    const int n_chunks = (L + a.chunk_tokens - 1) / a.chunk_tokens;
-    const int64_t stride = (int64_t)hq * (hd + 2);
-    const float *base = a.partials + ((int64_t)si * a.max_chunks * hq + qh) * (hd + 2);
-    float M = -INFINITY;
-    for (int ch = lane; ch < n_chunks; ch += 32) M = fmaxf(M, base[ch * stride]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    float S = 0.f;
-    for (int ch = lane; ch < n_chunks; ch += 32) {
-        const float m = base[ch * stride], s = base[ch * stride + 1];
-        S += (m == -INFINITY) ? 0.f : s * expf(m - M);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
-    float av[4] = {0.f, 0.f, 0.f, 0.f};  // channels lane, lane + 32, lane + 64, lane + 96
-#pragma unroll 4
-    for (int ch = 0; ch < n_chunks; ++ch) {
-        const float *part = base + ch * stride;
-        const float m = part[0];
-        const float w = (m == -INFINITY) ? 0.f : expf(m - M);
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (lane + 32 * j < hd) av[j] = fmaf(w, part[2 + lane + 32 * j], av[j]);
-    }
-    float c0 = 1.f, c1 = 0.f;
-    const T *vc = nullptr;
-    if (a.flags & KVCAR_INCLUDE_CURRENT_EXACT) {
+    const bool with_cur = (a.flags & KVCAR_INCLUDE_CURRENT_EXACT) != 0;
+    // current token: its operands do not depend on the partials
+    float qv[4] = {0.f, 0.f, 0.f, 0.f}, kv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
+    if (with_cur) {
         const int g = qh / (hq / a.hkv);
         const int W = a.hkv * hd;
         const T *kc = reinterpret_cast<const T *>(a.plan->cur[0][g]) + (int64_t)seq * W + a.plan->cur_head[0][g] * hd;
-        vc = reinterpret_cast<const T *>(a.plan->cur[1][g]) + (int64_t)seq * W + a.plan->cur_head[1][g] * hd;
+        const T *vc = reinterpret_cast<const T *>(a.plan->cur[1][g]) + (int64_t)seq * W + a.plan->cur_head[1][g] * hd;
         const T *qg = reinterpret_cast<const T *>(a.q) + ((int64_t)si * hq + qh) * hd;
-        float prod = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if (lane + 32 * j < hd) prod = fmaf(ld(qg + lane + 32 * j), ld(kc + lane + 32 * j), prod);
+            if (lane + 32 * j < hd) {
+                qv[j] = ld(qg + lane + 32 * j);
+                kv[j] = ld(kc + lane + 32 * j);
+                vv[j] = ld(vc + lane + 32 * j);
+            }
+    }
+    const int L = a.seq_len[seq];
+    const int n_chunks = (L + a.chunk_tokens - 1) / a.chunk_tokens;  // <= 32 (the launcher's choice)
+    const int64_t stride = (int64_t)hq * (hd + 2);
+    const float *base = a.partials + ((int64_t)si * a.max_chunks * hq + qh) * (hd + 2);
+    // lane c: tile c
+    float m_c = -INFINITY, s_c = 0.f;
+    if (lane < n_chunks) {
+        m_c = base[lane * stride];
+        s_c = base[lane * stride + 1];
+    }
+    // all weighted values: tile c, channels lane + 32 j
+    float pv[32][2];
+    const bool wide = hd > 64;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+        pv[c][0] = pv[c][1] = 0.f;
+        if (c < n_chunks) {
+            const float *part = base + c * stride + 2;
+            if (lane < hd) pv[c][0] = part[lane];
+            if (lane + 32 < hd) pv[c][1] = part[lane + 32];
+        }
+    }
+    float M = m_c;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    const float w_c = (m_c == -INFINITY) ? 0.f : expf(m_c - M);
+    float S = s_c * w_c;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
+    float av[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+        const float w = __shfl_sync(0xffffffffu, w_c, c);
+        av[0] = fmaf(w, pv[c][0], av[0]);
+        av[1] = fmaf(w, pv[c][1], av[1]);
+    }
+    if (wide) {  // head_dim above 64: channels 64.. in a second, plain pass
+        for (int c = 0; c < n_chunks; ++c) {
+            const float w = __shfl_sync(0xffffffffu, w_c, c);
+            const float *part = base + c * stride + 2;
+            if (lane + 64 < hd) av[2] = fmaf(w, part[lane + 64], av[2]);
+            if (lane + 96 < hd) av[3] = fmaf(w, part[lane + 96], av[3]);
+        }
+    }
+    float c0 = 1.f, c1 = 0.f;
+    if (with_cur) {
+        float prod = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) prod = fmaf(qv[j], kv[j], prod);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) prod += __shfl_xor_sync(0xffffffffu, prod, o);
         const float sc = prod * a.scale;
@@ -509,7 +540,7 @@ __global__ void __launch_bounds__(32 * CB_WARPS) combine_warp_kernel(const __gri
     for (int j = 0; j < 4; ++j) {
         const int c = lane + 32 * j;
         if (c < hd) {
-            const float acc = av[j] * c0 + (vc ? ld(vc + c) * c1 : 0.f);
+            const float acc = av[j] * c0 + vv[j] * c1;
             st(o + c, S > 0.f ? acc / S : 0.f);
         }
     }
@@ -565,10 +596,9 @@ cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int 
 }
 
 cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, int n_chunks, cudaStream_t st) {
-    // Many (sequence, query head) rows of few tiles each: one warp per row.  Otherwise a CTA per row, which merges
-    // a row's tiles in parallel (measured: 1024 rows x 16 tiles are 2 us per call faster with warps; 96 rows x
-    // 8 tiles and 384 rows x 33 tiles are faster with CTAs).
-    if (n_chunks <= 32 && a.hq * seqs.n >= 512) {
+    // At most 32 tiles per sequence: one warp per (sequence, query head) row, everything in two round trips.
+    // Longer sequences: a CTA per row, which walks a row's tiles in parallel.
+    if (n_chunks <= 32) {
         const int grid = (a.hq * seqs.n + CB_WARPS - 1) / CB_WARPS;
         if (dtype == KVCAR_F32)
             combine_warp_kernel<float><<<grid, 32 * CB_WARPS, 0, st>>>(a, seqs);
