@@ -246,6 +246,24 @@ def test_many_short_sequences_merge_one_warp_per_row(storage):
     _check_step(p.decode_step(seqs, 1, include_current=False), storage, f"warp merge, cached only, {storage}")
 
 
+@pytest.mark.parametrize("head_dim", [32, 128])
+def test_other_head_widths_take_the_generic_kernels(head_dim):
+    """Head widths other than 64 run on the generic kernels (fp32 and bf16 storage); 128 exercises the merge
+    kernels' upper channel half, 32 their idle lanes.  One sequence is long enough (33 tiles) for the
+    CTA-per-row merge, the others take the warp-per-row one."""
+    for storage in ("f32", "bf16"):
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=head_dim,
+                         latent_full=head_dim, batch=2, cached_tokens=0, decode_steps=1, reuse_frac=0.5,
+                         storage=storage)
+        for lens in ((200, 1), (4200, 130)):
+            pps = (max(lens) + 2 + w.page_tokens - 1) // w.page_tokens
+            p = Pair(w, max_seqs=2, max_pages=2 * pps, max_pages_per_seq=pps)
+            p.open([0, 1])
+            for s_, n in zip((0, 1), lens):
+                p.prefill([s_], n)
+            _check_step(p.decode_step([0, 1], 0), storage, f"head_dim {head_dim} {storage} {lens}")
+
+
 def test_fp32_stack_with_reuse_generic():
     """fp32 mode on a multi-layer stack with chains of reuse; 1e-4 absolute."""
     w = synth.scaled(synth.CONFIGS["c2"], n_layers=4, batch=2, storage="f32", reuse_frac=0.5)
