@@ -31,6 +31,15 @@
 // Operand staging.  16-KB places: a ring beside the hidden activations, plus, during
 // hidden-chunk jobs, the hidden slabs that hold no activations yet.
 //
+// Builds.  The kernel is a template over two properties of a launch, so that the shapes that need neither carry none
+// of the code:
+//   GMMA  more than two query heads per KV head: the scores and the weighted values of a group are small matrix
+//         products and run on the warp-level tensor op, fed straight from tensor memory in fragment layout;
+//         probabilities travel as bf16 rows, to the peer CTA by bulk copies that count their bytes on its barrier.
+//   SLAB  every hidden layer is one chunk (<= 256 columns): activations are handed to the second layer's products
+//         slab by slab, each source's scale/shift/bias block stays in shared memory, and the next pair's tiles,
+//         cache rows and queries are fetched while the current pair's last products run.
+//
 // Warp roles: warps 0 and 10 = TMA producers (both CTAs; they take alternate loads),
 // warp 1 = MMA issuer (leader CTA) and tensor-memory owner, warps 2-9 = epilogue (lane
 // quarter = warp % 4, column half = (warp-2) / 4).
