@@ -63,3 +63,32 @@ def test_scratch_too_small_is_refused():
     with pytest.raises(B.KvcarError) as e:
         B.head_l1_distance(2, 4, 64, B.BF16, x.data_ptr(), 64, scratch.data_ptr(), 4, out.data_ptr(), 0)
     assert e.value.status == 4          # KVCAR_ERR_WORKSPACE
+
+
+def test_reuse_table_from_distances_drives_the_cache():
+    """Alg. 2 end to end on synthetic activations: distances on the GPU, the closest heads chosen by the library,
+    the table handed to a cache context, and a decode step over that cache checked against the oracle, which gets
+    the table chosen by ITS OWN distance and choice functions (the two tables must be identical)."""
+    import kvcar_synth as synth
+    from kvcar_harness import Pair, assert_close
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=4, batch=2, cached_tokens=0, decode_steps=1, reuse_frac=0.0)
+    hkv, hd, L = w.n_kv_heads, w.head_dim, w.n_layers
+    tables = {}
+    for which, seed in (("k", 21), ("v", 22)):
+        x = _activations(L, 600, hkv, hd, seed=seed, dtype=torch.bfloat16)
+        got = _run(x, hkv, hd, B.BF16)
+        n_reuse = 5
+        lib_table = B.reuse_map_from_l1(got.ravel().tolist(), L, hkv, n_reuse)
+        want = orc.head_l1_distance(x.float().numpy().astype(np.float64), hkv)
+        oracle_table = orc.reuse_map_from_l1(want, n_reuse).tolist()
+        assert lib_table == oracle_table, which          # the distances differ by ~1e-7 relative: same ranking here
+        tables[which] = np.array(lib_table, dtype=np.int32)
+    assert (tables["k"] >= 0).sum() == 5 and not np.array_equal(tables["k"], tables["v"])
+    p = Pair(w, max_seqs=2, max_pages=12, max_pages_per_seq=6, src_k=tables["k"], src_v=tables["v"])
+    p.open([0, 1])
+    p.prefill([0], 300)
+    p.prefill([1], 129)
+    for l, (gpu, ref, rows) in p.decode_step([0, 1], 0).items():
+        assert_close(gpu[rows], ref, "bf16", f"layer {l}")
+    stored = sum(len(p.o.stored_heads(l, 0)) for l in range(L))
+    assert stored == L * hkv - 5                         # the five reused K heads store nothing
