@@ -31,17 +31,19 @@ def _prefill_device(p, w, seqs, n_tokens, seed, chunk=1024):
     p.s.ctx.sync_status(p.s.stream())
 
 
-def _run(w, sampled, steps=1):
+def _run(w, sampled, steps=1, fused=False, compress=True):
     pps = (w.cached_tokens + steps + w.page_tokens - 1) // w.page_tokens
-    p = Pair(w, max_seqs=w.batch, max_pages=w.batch * pps, max_pages_per_seq=pps, kernel=B.KERNEL_AUTO)
+    p = Pair(w, max_seqs=w.batch, max_pages=w.batch * pps, max_pages_per_seq=pps, kernel=B.KERNEL_AUTO,
+             compress=compress)
     p.oracle_seqs = set(sampled)
     seqs = list(range(w.batch))
     p.open(seqs)
     _prefill_device(p, w, seqs, w.cached_tokens, w.seed)
-    assert all(p.s.ctx.layer_kernel(l) == B.KERNEL_TENSOR for l in range(w.n_layers))
+    want_kernel = B.KERNEL_TENSOR if compress else B.KERNEL_RAW
+    assert all(p.s.ctx.layer_kernel(l) == want_kernel for l in range(w.n_layers))
     worst = 0.0
     for step in range(steps):
-        res = p.decode_step(seqs, step)
+        res = p.decode_step(seqs, step, fused=fused)
         for l, (got, ref, rows) in res.items():
             assert rows == sorted(sampled)
             err, _ = assert_close(got[rows], ref, w.storage, f"{w.name} step {step} layer {l}")
@@ -79,3 +81,18 @@ def test_config5_batch_sweep_point_sampled():
     sweep; many waves of clusters), first four layers; sequence 17 against the oracle."""
     w = synth.scaled(synth.with_batch(synth.CONFIGS["c5"], 32), n_layers=4)
     _run(w, [17], steps=1)
+
+
+def test_config5_largest_batch_single_call_step_sampled():
+    """The batch sweep's largest point: 256 sequences of 4096 cached tokens (8448 tiles, 57 tile pairs per
+    cluster), first two layers, each layer's step through the single-call entry point; the first and the last
+    sequence against the oracle."""
+    w = synth.scaled(synth.with_batch(synth.CONFIGS["c5"], 256), n_layers=2)
+    _run(w, [0, 255], steps=1, fused=True)
+
+
+def test_config3_uncompressed_twin_sampled():
+    """Raw K/V pages at the TinyLLaMA shape, full batch and length, first six layers (reuse redirects heads to
+    the lower layer's rows): the streaming kernel with 8 query heads per KV head."""
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=6)
+    _run(w, [5, 31], steps=1, compress=False)
