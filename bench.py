@@ -54,6 +54,9 @@ def parse():
     ap.add_argument("--head-l1", action="store_true",
                     help="instead of the decode step: time Alg. 2's head-distance reduction on K rows shaped like "
                          "the workload (layers x batch*cached_tokens x KV width) and print its own JSON line")
+    ap.add_argument("--prefill", action="store_true",
+                    help="instead of the decode step: time the bulk encoder + append of 1024 tokens per sequence, on the "
+                         "tensor cores (kvcar_encode_append_tensor) and on the CUDA cores, and print its own JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle sample")
@@ -399,10 +402,59 @@ def run_head_l1(args):
                       "max_rel_err_vs_oracle_on_256_rows": err, "gpu_launches": 2 * K_}))
 
 
+def run_prefill(args):
+    """Bulk encoder + append: one call per layer of 1024 new tokens per sequence."""
+    import torch
+    w = workload_of(args)
+    chunk = 1024
+    K_, W_ = args.steps, max(args.warmup, 3)
+    peaks = measured_peaks()
+    out = {}
+    for name in ("tensor", "cuda_cores"):
+        sess, src, aes = build_session(synth.scaled(w, cached_tokens=0), args, torch, chunk * (K_ + W_) + 8)
+        seqs = list(range(w.batch))
+        for q in seqs:
+            sess.ctx.seq_open(q)
+        g = torch.Generator(device="cuda").manual_seed(w.seed)
+        k = torch.randn(w.batch, chunk, w.kv_width, generator=g, device="cuda").to(torch.bfloat16)
+        v = torch.randn(w.batch, chunk, w.kv_width, generator=g, device="cuda").to(torch.bfloat16)
+        stream = sess.stream()
+        call = sess.ctx.encode_append_tensor if name == "tensor" else sess.ctx.encode_append
+        ms = []
+        for i in range(W_ + K_):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for l in range(w.n_layers):
+                call(l, seqs, chunk, k.data_ptr(), v.data_ptr(), stream)
+            b.record()
+            sess.ctx.advance(seqs, chunk, stream)
+            torch.cuda.synchronize()
+            if i >= W_:
+                ms.append(a.elapsed_time(b))
+        sess.ctx.sync_status(stream)
+        out[name] = sum(ms) / len(ms)
+        flops = 0.0
+        for (l, which), ae in aes.items():
+            flops += 2.0 * (ae["in_dim"] * ae["hidden"] + ae["hidden"] * ae["latent"]) * w.batch * chunk
+        del sess
+    tf = flops / (out["tensor"] / 1e3) / 1e12
+    print(json.dumps({"metric": "prefill tokens/s (bulk encoder + append, all layers)", "value": w.batch * chunk / (out["tensor"] / 1e3),
+                      "unit": "tokens/s", "n_gpus": 1, "steps": K_, "warmup": W_, "ms_per_step": out["tensor"],
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": w.name + "_prefill", "layers": w.n_layers, "rows_per_call": w.batch * chunk},
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                   "frac": tf / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"] + " (burst)",
+                                   "algorithmic_flops_per_step": flops},
+                      "cuda_core_encoder_ms_per_step": out["cuda_cores"]}))
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.prefill:
+        run_prefill(args)
         return
     if args.head_l1:
         run_head_l1(args)

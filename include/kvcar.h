@@ -171,6 +171,21 @@ kvcar_status kvcar_reserve(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, 
 kvcar_status kvcar_encode_append(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                  int32_t n_tokens, const void *k, const void *v, void *stream);
 
+/*
+ * kvcar_encode_append on the tensor cores, for many tokens per sequence (cache
+ * prefill): same arguments, same rows written, same current-token rows (Sec.
+ * "Network Architecture", the encoder of the appended key and value vectors).
+ * The two fully connected layers run as tiled bf16 products with fp32
+ * accumulation, so the hidden activations pass through bf16 between them
+ * (kvcar_encode_append keeps them in fp32): a latent may differ from that
+ * call's by a few bf16 steps of the row's scale.  Only bf16 storage, 64-wide
+ * heads, and layers whose K and V both have an autoencoder with hidden and
+ * latent widths that are multiples of 16 (else KVCAR_ERR_UNSUPPORTED, nothing
+ * written).  Other errors as kvcar_encode_append.
+ */
+kvcar_status kvcar_encode_append_tensor(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                        int32_t n_tokens, const void *k, const void *v, void *stream);
+
 /* seq_len += n_tokens for the listed sequences (host mirror now, device copy in
  * stream order). */
 kvcar_status kvcar_advance(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens, void *stream);

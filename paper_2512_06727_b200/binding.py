@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "STATE", 3: "OOM_PAGES", 4: "WORKS
 EXPORTS = [
     "kvcar_create", "kvcar_destroy", "kvcar_set_reuse_map", "kvcar_set_autoencoder", "kvcar_required_bytes",
     "kvcar_bind_memory", "kvcar_set_kernel", "kvcar_seq_open", "kvcar_seq_close", "kvcar_reserve",
-    "kvcar_encode_append", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
+    "kvcar_encode_append", "kvcar_encode_append_tensor", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
     "kvcar_step_layer", "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
@@ -92,6 +92,7 @@ def _load() -> C.CDLL:
         "kvcar_seq_close": [vp, i32],
         "kvcar_reserve": [vp, ip, i32, i32],
         "kvcar_encode_append": [vp, i32, ip, i32, i32, vp, vp, vp],
+        "kvcar_encode_append_tensor": [vp, i32, ip, i32, i32, vp, vp, vp],
         "kvcar_advance": [vp, ip, i32, i32, vp],
         "kvcar_decode_attention": [vp, i32, ip, i32, vp, vp, u32, vp],
         "kvcar_decode_attention_static": [vp, i32, ip, i32, vp, vp, u32, vp],
@@ -244,6 +245,10 @@ class Context:
     # -- hot path ----------------------------------------------------------
     def encode_append(self, layer: int, seqs: Sequence[int], n_tokens: int, k: int, v: int, stream: int = 0):
         self._check(self.lib.kvcar_encode_append(self._h, layer, self._seqs(seqs), len(seqs), n_tokens, k, v, stream))
+
+    def encode_append_tensor(self, layer: int, seqs: Sequence[int], n_tokens: int, k: int, v: int, stream: int = 0):
+        self._check(self.lib.kvcar_encode_append_tensor(self._h, layer, self._seqs(seqs), len(seqs), n_tokens, k, v,
+                                                        stream))
 
     def advance(self, seqs: Sequence[int], n_tokens: int, stream: int = 0):
         self._check(self.lib.kvcar_advance(self._h, self._seqs(seqs), len(seqs), n_tokens, stream))

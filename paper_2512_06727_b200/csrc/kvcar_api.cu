@@ -55,7 +55,8 @@ struct kvcar_ctx {
     std::vector<int> width;                 // elements per row
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
     size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
-    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0;  // inside workspace
+    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0, pfhid_off = 0;  // inside workspace
+    std::vector<EncPlan> enc_host;  // the device's EncPlan table, host copy (tensor-core prefill builds tensor maps from it)
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
     std::vector<LayerPlan> plans_host;
@@ -171,6 +172,8 @@ void compute_layout(kvcar_ctx *c) {
     s = align_up(s + (size_t)2 * nb * c->max_m * sizeof(float), 256);
     c->kvsplit_off = s;  // probabilities handed from K clusters to V clusters (tensor-core kernel, small grids)
     s = align_up(s + tc_split_bytes(g), 256);
+    c->pfhid_off = s;  // bf16 hidden activations between the two launches of the tensor-core prefill
+    if (g.storage == KVCAR_BF16 && c->max_m > 0) s = align_up(s + prefill_tc_scratch_bytes(c->max_m), 256);
     c->ws_bytes = s;
 }
 
@@ -531,6 +534,7 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
         }
     }
     memcpy(&img[c->enc_off], enc.data(), enc.size() * sizeof(EncPlan));
+    c->enc_host = enc;
 
     cudaError_t e = cudaMemcpyAsync(c->weights, img.data(), img.size(), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->part_off, st);  // tables, lengths, status
@@ -640,6 +644,52 @@ static kvcar_status enqueue_encode(kvcar_ctx *c, int32_t layer, const int32_t *s
                              : launch_encode_generic(a, sl, c->cfg.storage, c->max_in, c->max_m, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "encode launch");
     c->launches += split_ok ? 2 : 1;
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_encode_append_tensor(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs,
+                                        int32_t n_tokens, const void *k, const void *v, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (layer < 0 || layer >= c->cfg.n_layers || !k || !v || n_tokens <= 0)
+        return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer, pointer or token count");
+    if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "k/v must be 16-byte aligned");
+    const kvcar_config &g = c->cfg;
+    if (g.storage != KVCAR_BF16 || g.head_dim != 64)
+        return fail(c, KVCAR_ERR_UNSUPPORTED, "the tensor-core encoder takes bf16 storage and 64-wide heads");
+    for (int w = 0; w < 2; ++w) {
+        const AEHost &ae = c->ae[layer * 2 + w];
+        if (!ae.set || ae.hidden % 16 || ae.latent % 16 || ae.hidden > 1024 || ae.latent > 1024)
+            return fail(c, KVCAR_ERR_UNSUPPORTED,
+                        "the tensor-core encoder needs an autoencoder for K and for V with widths that are multiples of 16");
+    }
+    if ((int64_t)n_seqs * n_tokens > 0x7fffffff) return fail(c, KVCAR_ERR_INVALID_ARG, "too many rows");
+    kvcar_status s = reserve_pages(c, seqs, n_seqs, n_tokens);
+    if (s != KVCAR_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    s = flush_tables(c, st);
+    if (s != KVCAR_OK) return s;
+    PrefillTcArgs a{};
+    a.plan_dev = reinterpret_cast<const EncPlan *>(c->weights + c->enc_off) + layer * 2;
+    a.plan_host = c->enc_host.data() + layer * 2;
+    a.block_table = reinterpret_cast<const int32_t *>(c->ws + c->bt_off);
+    a.seq_len = reinterpret_cast<const int32_t *>(c->ws + c->len_off);
+    a.status = reinterpret_cast<int32_t *>(c->ws + c->status_off);
+    a.src[0] = k;
+    a.src[1] = v;
+    a.hid = c->ws + c->pfhid_off;
+    a.max_m = c->max_m;
+    a.max_pages_per_seq = g.max_pages_per_seq;
+    a.page_tokens = g.page_tokens;
+    a.n_tokens = n_tokens;
+    a.kv_width = g.n_kv_heads * g.head_dim;
+    SeqList sl;
+    sl.n = n_seqs;
+    memcpy(sl.id, seqs, (size_t)n_seqs * 4);
+    cudaError_t e = launch_prefill_tc(a, sl, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "tensor-core encoder launch");
+    c->launches += 2 * (((int64_t)n_seqs * n_tokens + PREFILL_TC_ROWS - 1) / PREFILL_TC_ROWS);
     return KVCAR_OK;
 }
 

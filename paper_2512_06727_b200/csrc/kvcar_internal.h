@@ -114,4 +114,22 @@ cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtyp
 cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, int n_chunks, cudaStream_t st);
 size_t decode_generic_smem(int hq, int hd, int max_d, int max_m);
 
+// Bulk encoder + append on the tensor cores (kvcar_prefill_tc.cu): bf16 storage, both K and V of the layer with an
+// autoencoder, head_dim 64, hidden and latent widths multiples of 16.  Rows are worked through in blocks of
+// PREFILL_TC_ROWS; `hid` is a bf16 scratch of prefill_tc_scratch_bytes(max hidden width) bytes.
+constexpr int PREFILL_TC_ROWS = 8192;
+struct PrefillTcArgs {
+    const EncPlan *plan_dev;    // this layer's [K, V] plans on the device
+    const EncPlan *plan_host;   // the same two plans, host copy (widths and weight pointers for the tensor maps)
+    const int32_t *block_table;
+    const int32_t *seq_len;
+    int32_t *status;
+    const void *src[2];         // the caller's K and V rows [n_seqs * n_tokens][kv_width]
+    void *hid;
+    int32_t max_m;
+    int32_t max_pages_per_seq, page_tokens, n_tokens, kv_width;
+};
+size_t prefill_tc_scratch_bytes(int max_m);
+cudaError_t launch_prefill_tc(const PrefillTcArgs &a, const SeqList &seqs, cudaStream_t st);
+
 }  // namespace kvcar
