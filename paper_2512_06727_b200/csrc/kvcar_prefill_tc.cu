@@ -22,7 +22,7 @@ namespace {
 
 constexpr int PF_M = 128;          // rows per CTA
 constexpr int PF_N = 256;          // columns per CTA at most
-constexpr int PF_STAGES = 4;
+constexpr int PF_STAGES = 2;       // two CTAs share an SM: one's epilogue runs under the other's products
 constexpr int PF_A_BYTES = PF_M * 128;   // one 64-wide K slab of the row tile (bf16, 128-byte rows)
 constexpr int PF_B_BYTES = PF_N * 128;
 constexpr int PF_STAGE_BYTES = PF_A_BYTES + PF_B_BYTES;
@@ -131,12 +131,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // grid = (row tiles, column tiles, 2 [K, V]); STAGE 1 or 2 as in the file header
 template <int STAGE>
-__global__ void __launch_bounds__(PF_THREADS, 1)
+__global__ void __launch_bounds__(PF_THREADS, 2)
     prefill_fc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                       const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
                       const __grid_constant__ PfArgs a, const __grid_constant__ SeqList seqs) {
     extern __shared__ uint8_t pf_smem[];
     __shared__ uint32_t tmem_slot;
+    __shared__ __align__(16) float prm[2][PF_N];  // this tile's columns of scale and shift (stage 1) or bias (stage 2)
     const int which = blockIdx.z;
     const EncPlan &pl = a.plan[which];
     const int kdim = STAGE == 1 ? pl.in_dim : pl.m, ndim = STAGE == 1 ? pl.m : pl.d;
@@ -229,8 +230,15 @@ __global__ void __launch_bounds__(PF_THREADS, 1)
                 tok % a.page_tokens;
             dst = reinterpret_cast<__nv_bfloat16 *>(pl.pool) + prow * pl.width + n0;
         }
-        const float *p0 = STAGE == 1 ? pl.s1 + n0 : pl.b2 + n0;
-        const float *p1 = STAGE == 1 ? pl.t1 + n0 : nullptr;
+        {
+            const float *g0 = STAGE == 1 ? pl.s1 + n0 : pl.b2 + n0;
+            const float *g1 = STAGE == 1 ? pl.t1 + n0 : nullptr;
+            for (int i = threadIdx.x - 64; i < nt; i += 128) {
+                prm[0][i] = g0[i];
+                if (STAGE == 1) prm[1][i] = g1[i];
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
         const float slope = pl.slope;
         if (mbar_wait(bar_acc, 0, a.status, 0x403)) {
             tc_fence_after();
@@ -243,15 +251,21 @@ __global__ void __launch_bounds__(PF_THREADS, 1)
                 for (int c8 = 0; c8 < 4; ++c8) {
                     const int c = 32 * g + 8 * c8;
                     if (c >= nt) break;
-                    float o[8];
+                    float o[8], pa[8], pb[8];
+                    *reinterpret_cast<float4 *>(pa) = *reinterpret_cast<const float4 *>(&prm[0][c]);
+                    *reinterpret_cast<float4 *>(pa + 4) = *reinterpret_cast<const float4 *>(&prm[0][c + 4]);
+                    if (STAGE == 1) {
+                        *reinterpret_cast<float4 *>(pb) = *reinterpret_cast<const float4 *>(&prm[1][c]);
+                        *reinterpret_cast<float4 *>(pb + 4) = *reinterpret_cast<const float4 *>(&prm[1][c + 4]);
+                    }
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const float x = v[8 * c8 + e];
                         if (STAGE == 1) {
-                            const float y = fmaf(x, __ldg(p0 + c + e), __ldg(p1 + c + e));
+                            const float y = fmaf(x, pa[e], pb[e]);
                             o[e] = y > 0.f ? y : y * slope;
                         } else {
-                            o[e] = x + __ldg(p0 + c + e);
+                            o[e] = x + pa[e];
                         }
                     }
                     *reinterpret_cast<uint4 *>(dst + c) =
