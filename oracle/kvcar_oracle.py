@@ -58,10 +58,13 @@ def round_to_storage(x: np.ndarray, storage: str) -> np.ndarray:
         return np.asarray(x, dtype=np.float64).astype(np.float32).astype(np.float64)
     if storage == "bf16":
         return round_to_bf16(x)
+    if storage == "int8":
+        return int8_rows(x)
     raise ValueError(storage)
 
 
-STORAGE_BYTES = {"exact": 8, "f32": 4, "bf16": 2}
+STORAGE_BYTES = {"exact": 8, "f32": 4, "bf16": 2, "int8": 1}
+INT8_ROW_PARAM_BYTES = 8   # scale and zero-point (fp32 each) kept beside every int8 row
 
 
 # --------------------------------------------------------------------------
@@ -86,6 +89,23 @@ def int8_quantize(x: np.ndarray) -> Tuple[np.ndarray, float, float]:
 def int8_dequantize(q: np.ndarray, scale: float, zeropoint: float) -> np.ndarray:
     """Eq. 4, last line: (q - zeropoint)/scale."""
     return (np.asarray(q, dtype=np.float64) - zeropoint) / scale
+
+
+def int8_rows(z: np.ndarray) -> np.ndarray:
+    """Latent rows as an int8 cache would return them (Sec. "Quantization", Eq. 4 applied on top of the
+    autoencoder as in Table 5): every row is quantised with its own scale and zero-point - the paper does not
+    state the granularity; a token's row is the unit that is written and read together - and dequantised again.
+    A row of equal values has no range to scale and is kept as it is."""
+    z = np.asarray(z, dtype=np.float64)
+    out = np.empty_like(z)
+    flat_in, flat_out = z.reshape(-1, z.shape[-1]), out.reshape(-1, z.shape[-1])
+    for i, row in enumerate(flat_in):
+        if row.max() == row.min():
+            flat_out[i] = row
+        else:
+            q, scale, zp = int8_quantize(row)
+            flat_out[i] = int8_dequantize(q, scale, zp)
+    return out
 
 
 # --------------------------------------------------------------------------
@@ -347,5 +367,8 @@ class KVCAROracle:
         compression and reuse, bytes without either)."""
         b = STORAGE_BYTES[self.storage]
         comp = sum(self.stored_width(l, w) for l in range(self.n_layers) for w in (K, V)) * b
+        if self.storage == "int8":   # per stored row: its scale and zero-point; the uncompressed reference is 16-bit
+            comp += INT8_ROW_PARAM_BYTES * sum(1 for l in range(self.n_layers) for w in (K, V) if self.stored_width(l, w))
+            b = 2
         full = 2 * self.n_layers * self.hkv * self.hd * b
         return float(comp), float(full)

@@ -598,3 +598,33 @@ def test_reuse_map_from_l1_picks_the_closest_heads():
     o = KVCAROracle(4, 3, 3, 4, page_tokens=2, max_seqs=1, max_pages=4, storage="exact")
     o.set_reuse_map(four, four)
     assert o.resolve(3, 0, K)[:2] == (1, 0)
+
+
+def test_int8_latent_rows_stay_within_half_a_step():
+    """Eq. 4 per cached row (the storage mode an int8 latent cache would have): every value comes back within
+    half a quantisation step of itself, the row's extremes within one step, a constant row unchanged, and the
+    cache accounting charges one byte per element plus the row's scale and zero-point."""
+    rng = np.random.default_rng(9)
+    z = rng.normal(size=(5, 7, 48)) * rng.uniform(0.1, 10.0, size=(5, 7, 1))
+    z[2, 3] = 1.25                                              # a row of equal values
+    back = orc.int8_rows(z)
+    step = (z.max(axis=-1, keepdims=True) - z.min(axis=-1, keepdims=True)) / 255.0
+    assert np.all(np.abs(back - z) <= 0.5 * step + 1e-12)
+    assert np.array_equal(back[2, 3], z[2, 3])
+    row = z[0, 0]
+    q, scale, zp = orc.int8_quantize(row)
+    assert q.min() >= -128 and q.max() <= 127 and np.all(q == np.rint(q))
+    assert abs(orc.int8_dequantize(q, scale, zp).max() - row.max()) <= step[0, 0, 0]
+    # rows are independent: quantising a row alone or inside a batch gives the same values
+    assert np.array_equal(orc.int8_rows(z[1, 2][None])[0], back[1, 2])
+    # the cache model stores them and accounts for them
+    o = KVCAROracle(2, 2, 2, 4, page_tokens=2, max_seqs=1, max_pages=4, storage="int8")
+    o.set_reuse_map([-1, -1, 0, -1], [-1, -1, -1, -1])          # layer 1 K head 0 reuses layer 0
+    comp, full = o.cache_bytes_per_token()
+    assert comp == (8 + 8 + 4 + 8) * 1 + 4 * 8                  # widths 8, 8, 4, 8 at one byte + four rows' parameters
+    assert full == 2 * 2 * 8 * 2                                # against 16-bit raw K/V
+    o.seq_open(0)
+    k = rng.normal(size=(1, 3, 8)); v = rng.normal(size=(1, 3, 8))
+    o.encode_append(0, [0], 3, k, v)
+    stored = o._pool(0, K)[[o.locate(0, t)[1] for t in range(3)]]
+    np.testing.assert_array_equal(stored, orc.int8_rows(k[0]))
