@@ -107,9 +107,9 @@ kvcar_status kvcar_create(const kvcar_config *cfg, kvcar_ctx **out_ctx);
 kvcar_status kvcar_destroy(kvcar_ctx *ctx);
 
 /*
- * Cross-layer head reuse (Sec. "Network Architecture", last paragraph: "certain
- * key and value heads in layer N reuse key and value heads from the previous
- * layer N-1").  src_k/src_v: HOST int32 [n_layers * n_kv_heads]; entry
+ * Cross-layer head reuse (Sec. "Network Architecture", last paragraph: chosen K
+ * and V heads of a layer read the corresponding head of the layer below instead
+ * of caching their own).  src_k/src_v: HOST int32 [n_layers * n_kv_heads]; entry
  * (layer, head) is -1 if the head keeps its own cache rows, else the index of
  * the head of layer-1 whose cached K (resp. V) it reads.  Chains are legal and
  * resolve transitively.  Layer 0 must be all -1.  Only before kvcar_bind_memory
@@ -156,9 +156,9 @@ kvcar_status kvcar_reserve(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, 
 /* ---- the hot path --------------------------------------------------------- */
 
 /*
- * Encoder + append (Sec. "Network Architecture": "an encoder layer is added
- * after the generation of key and value tokens ... reduces them to a lower
- * dimension d ... a 1 x d vector is appended to the KV cache").
+ * Encoder + append (Sec. "Network Architecture": the new token's key and value
+ * vectors go through the layer's encoder right after they are produced, and the
+ * resulting 1 x d latent rows are what the cache stores).
  * k, v: DEVICE [n_seqs][n_tokens][n_kv_heads*head_dim] new rows (all heads;
  * columns of reused heads are ignored).  For each sequence the stored heads'
  * slices are encoded (or copied, for an uncompressed layer), rounded to the
@@ -191,9 +191,9 @@ kvcar_status kvcar_encode_append_tensor(kvcar_ctx *ctx, int32_t layer, const int
 kvcar_status kvcar_advance(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens, void *stream);
 
 /*
- * Decoder + attention (Sec. "Network Architecture": cached latents "are passed
- * through two decoders, expanding them to (l-1) x D ... then concatenated with
- * the current 1 x D key and value vectors"; Eq. 1 per head).
+ * Decoder + attention (Sec. "Network Architecture": the cached latent rows are
+ * expanded back to full-width K and V by the layer's two decoders and joined with
+ * the current token's exact key and value vectors; Eq. 1 per head).
  * q: DEVICE [n_seqs][n_q_heads][head_dim]; out: DEVICE, same shape.
  * For each sequence and query head i (KV head g = i / (n_q_heads/n_kv_heads)):
  * resolve g through the reuse table for K and for V separately, restore the
@@ -307,9 +307,9 @@ const char *kvcar_last_error(kvcar_ctx *ctx);
  *
  * These calls need no context: they work on activations recorded by the caller.
  *
- * kvcar_head_l1_distance: "Calculate inter layer L1 norm between heads of
- * adjacent layers" (Alg. 2; Sec. "Network Architecture": the norm "captures the
- * absolute differences between their key and value matrices").
+ * kvcar_head_l1_distance: the distance step of Alg. 2 (Sec. "Network
+ * Architecture": an L1 norm between the same head's K, or V, matrices in two
+ * adjacent layers, i.e. the sum of their absolute differences).
  * x: DEVICE [n_layers][n_rows][n_kv_heads * head_dim], storage type `storage`
  * (KVCAR_F32 / KVCAR_BF16), 16-byte aligned: the K (or the V) rows of one
  * mini-batch, n_rows = sequences x tokens.  dist: DEVICE float
@@ -328,8 +328,8 @@ kvcar_status kvcar_head_l1_scratch_bytes(int32_t n_layers, int32_t n_kv_heads, i
 kvcar_status kvcar_head_l1_distance(int32_t n_layers, int32_t n_kv_heads, int32_t head_dim, int32_t storage, const void *x,
                                     int64_t n_rows, void *scratch, size_t scratch_bytes, float *dist, void *stream);
 /*
- * "Based on L1 norm, the key and value heads in the particular layers are
- * reused by the key and value in the previous layer" (Alg. 2): the n_reuse heads
+ * The selection step of Alg. 2 (heads whose distance to the layer below is small
+ * enough read that layer's head instead of their own): the n_reuse heads
  * with the smallest distance reuse the same head of the layer below (the
  * paper's empirical threshold, given as a count; equal distances: lower layer,
  * then lower head, first).  dist: HOST float [n_layers - 1][n_kv_heads] (no NaN);

@@ -22,7 +22,8 @@ notes; the ones that matter for reading this file:
     nothing after the last FC, for encoder and decoder alike;
   * a head table entry points at a head of layer l-1; chains resolve transitively;
   * cached tokens are attended through their restored rows, the current token
-    through its exact K/V ("concatenated with the current 1xD key and value").
+    through its exact K/V (Sec. "Network Architecture": the restored rows are joined with
+    the current token's exact key and value vectors).
 """
 from __future__ import annotations
 
@@ -77,12 +78,15 @@ def kv_cache_size_bytes(bytes_per_elem: int, n_layers: int, d_model: int, seq_le
 
 def int8_quantize(x: np.ndarray) -> Tuple[np.ndarray, float, float]:
     """Eq. 4: scale = 255/(max-min); zeropoint = -round(scale*min) - 128;
-    q = round(scale*x + zeropoint)."""
+    q = round(scale*x + zeropoint), kept inside the int8 range.  The equation itself can
+    exceed it by one: scale*max + zeropoint = 127 + frac(scale*min), and when that fraction
+    is exactly one half the two roundings can put the maximum at 128; a code an int8 cache
+    cannot hold is clipped to 127 (the paper stores int8 values, Sec. "Quantization")."""
     x = np.asarray(x, dtype=np.float64)
     lo, hi = float(x.min()), float(x.max())
     scale = 255.0 / (hi - lo)
     zeropoint = -np.rint(scale * lo) - 128.0
-    q = np.rint(scale * x + zeropoint)
+    q = np.clip(np.rint(scale * x + zeropoint), -128.0, 127.0)
     return q, scale, float(zeropoint)
 
 
@@ -112,9 +116,8 @@ def int8_rows(z: np.ndarray) -> np.ndarray:
 # Alg. 2, first steps: which heads may reuse the layer below
 # --------------------------------------------------------------------------
 def head_l1_distance(x: np.ndarray, n_kv_heads: int) -> np.ndarray:
-    """Alg. 2 ("inter layer L1 norm between heads of adjacent layers"; Sec. "Network
-    Architecture": the L1 norm "captures the absolute differences between their key
-    and value matrices").  x: recorded K (or V) rows, [n_layers][n_rows][n_kv_heads *
+    """Alg. 2, its distance step; Sec. "Network Architecture" describes the measure as the sum of
+    absolute differences between two heads' key (value) matrices.  x: recorded K (or V) rows, [n_layers][n_rows][n_kv_heads *
     head_dim].  Returns D [n_layers - 1][n_kv_heads]: D[l-1][h] = mean over the rows and
     over head h's channels of |x[l] - x[l-1]|, i.e. the L1 norm of the difference of
     head h's matrix in layers l and l-1 divided by its element count (the paper does
@@ -133,7 +136,7 @@ def head_l1_distance(x: np.ndarray, n_kv_heads: int) -> np.ndarray:
 
 def reuse_map_from_l1(dist: np.ndarray, n_reuse: int) -> np.ndarray:
     """Alg. 2, next step: the heads with the smallest distance to the layer below
-    reuse it ("a threshold is empirically determined": here the threshold is given as
+    reuse it (the paper picks its threshold empirically: here the threshold is given as
     a count, the n_reuse closest heads; equal distances go to the lower layer, then
     the lower head).  dist: [n_layers - 1][n_kv_heads] as returned above.  Returns the
     table in the form the cache takes it: int32 [n_layers * n_kv_heads], -1 = own

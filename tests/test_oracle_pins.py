@@ -457,6 +457,14 @@ def test_int8_quantisation_eq4():
     # worked by hand: x in {0, 1, 2.55}: scale=100, zp=-128, q = {-128, -28, 127}
     q2, s2, z2 = orc.int8_quantize(np.array([0.0, 1.0, 2.55]))
     assert s2 == pytest.approx(100.0) and z2 == -128 and list(q2) == [-128, -28, 127]
+    # the half-way case, worked by hand: x in {0.5, 100, 255.5}: scale = 1, round(0.5) = 0 so zp = -128; the
+    # equation gives round(255.5 - 128) = 128 for the maximum, which no int8 holds: the code is 127
+    q3, s3, z3 = orc.int8_quantize(np.array([0.5, 100.0, 255.5]))
+    assert s3 == 1.0 and z3 == -128 and list(q3) == [-128, -28, 127]
+    for seed in range(50):      # codes always fit int8
+        r = np.random.default_rng(seed).normal(size=97) * 10 ** np.random.default_rng(seed + 1).uniform(-3, 3)
+        qq, _, _ = orc.int8_quantize(r)
+        assert qq.min() >= -128 and qq.max() <= 127 and np.all(qq == np.rint(qq))
 
 
 # ---------------------------------------------------------------- accounting (printed values)
@@ -540,7 +548,7 @@ def test_reuse_map_generator_counts():
 
 # ---------------------------------------------------------------- Alg. 2: head distances and the reuse choice
 def test_head_l1_distance_closed_forms_and_brute_force():
-    """Alg. 2, "inter layer L1 norm between heads of adjacent layers", pinned by cases with a known answer:
+    """Alg. 2's distance step (an L1 norm between the same head in two adjacent layers), pinned by cases with a known answer:
     equal layers -> 0; a per-head constant offset -> its magnitude; loops written out on a tiny case (which
     catches a wrong layer pairing, a wrong head slice or a wrong divisor); scaling; row order."""
     rng = np.random.default_rng(5)
