@@ -30,10 +30,6 @@ if ROOT not in sys.path:
 
 import kvcar_synth as synth  # noqa: E402
 
-# DRAM bytes (read + write) per decode_pair_kernel launch from the ncu capture summarised in
-# profiles/decode_pair_kernel_c2.md (mean of two layers); only for the workload and kernel it was taken on
-NCU_TRAFFIC_BYTES = {("c2_gpt2s_12l_b8_L1024", "auto", False): 27.25e6}
-
 METRIC = "decode tokens/s over latent KV cache"
 UNIT = "tokens/s"
 
@@ -41,10 +37,11 @@ UNIT = "tokens/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--steps", type=int, default=12)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
-    ap.add_argument("--batch", type=int, default=None, help="override the batch (config 5 sweep)")
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override the batch (config 5 is the batch sweep; its default here is the largest point, 256)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tensor"])
     ap.add_argument("--uncompressed", action="store_true", help="raw K/V pages (the uncompressed twin)")
@@ -57,6 +54,10 @@ def parse():
     ap.add_argument("--prefill", action="store_true",
                     help="instead of the decode step: time the bulk encoder + append of 1024 tokens per sequence, on the "
                          "tensor cores (kvcar_encode_append_tensor) and on the CUDA cores, and print its own JSON line")
+    ap.add_argument("--capacity", action="store_true",
+                    help="instead of the decode step: longest sequence that fits per batch size at 0/25/50/75 %% compression from the\n"
+                         "library's own bytes-per-token accounting, plus one batch actually held in memory compressed vs raw")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle sample")
@@ -65,8 +66,9 @@ def parse():
 
 def workload_of(args) -> synth.Workload:
     w = synth.CONFIGS[args.workload]
-    if args.batch:
-        w = synth.with_batch(w, args.batch)
+    batch = args.batch or (256 if args.workload == "c5" else None)
+    if batch:
+        w = synth.with_batch(w, batch)
     return w
 
 
@@ -343,8 +345,10 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "batch": w.batch, "cached_tokens": w.cached_tokens,
-                       "layers": w.n_layers, "storage": w.storage},
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "cached_tokens": w.cached_tokens,
+                       "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+                       "latent_full": w.latent_full, "reuse_frac": w.reuse_frac, "page_tokens": w.page_tokens,
+                       "storage": w.storage},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -402,6 +406,86 @@ def run_head_l1(args):
                       "max_rel_err_vs_oracle_on_256_rows": err, "gpu_launches": 2 * K_}))
 
 
+def run_capacity(args):
+    """The B200 counterpart of the paper's Fig. 2 / Fig. 3 (Sec. "System Evaluation"): how long a sequence fits per
+    batch size at 0 / 25 / 50 / 75 % cache compression, from the library's own bytes-per-token accounting, and one
+    batch at 4096 tokens actually held in device memory, compressed (autoencoder 2x + the workload's reuse map) and raw."""
+    import torch
+    from paper_2512_06727_b200 import binding as B
+    free_b, total_b = torch.cuda.mem_get_info()
+    budget = int(free_b * 0.85)          # leave room for q/k/v, weights and the framework
+    out = {"metric": "longest sequence that fits (tokens) per batch size", "unit": "tokens", "data": "accounting",
+           "device_free_bytes": free_b, "device_total_bytes": total_b, "budget_bytes": budget, "curves": [], "held": []}
+
+    def bytes_per_token(w, level):
+        """level: fraction of the cache removed by autoencoders alone (no reuse), Table 2 style."""
+        ctx = B.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, 1, 1, 1,
+                        B.BF16 if w.storage == "bf16" else B.F32)
+        none = np.full(w.n_layers * w.n_kv_heads, -1, dtype=np.int32)
+        ctx.set_reuse_map(none, none)
+        if level > 0:
+            # 25 %: latent = half the width in half the layers; 50 %: in all layers; 75 %: a quarter of the width in all
+            layers = range(w.n_layers // 2) if level == 0.25 else range(w.n_layers)
+            lat_per_head = w.head_dim // 4 if level == 0.75 else w.head_dim // 2
+            for l in layers:
+                for which in (0, 1):
+                    in_dim, hidden, latent = synth.ae_dims(w.n_kv_heads, w.head_dim, lat_per_head)
+                    ctx.set_autoencoder(l, which, synth.make_autoencoder(in_dim, hidden, latent, w.seed, l, which,
+                                                                         storage=w.storage))
+        comp, full = ctx.cache_bytes_per_token()
+        return comp, full
+
+    for name in ("c5", "c3"):
+        w = synth.CONFIGS[name]
+        for level in (0.0, 0.25, 0.5, 0.75):
+            comp, full = bytes_per_token(w, level)
+            row = {"shape": "GPT-2-small 12x12x64" if name == "c5" else "TinyLLaMA 22 layers, 4 KV heads x 64",
+                   "compression": level, "cache_bytes_per_token": comp, "saved": 1.0 - comp / full, "max_tokens": {}}
+            for b in (1, 8, 16, 32, 64, 128, 256):
+                row["max_tokens"][str(b)] = int(budget // (b * comp))
+            out["curves"].append(row)
+
+    # one batch at 4096 tokens held for real: the workload's own configuration (autoencoders + reuse map) and its raw twin
+    w = synth.CONFIGS["c5"]
+    from paper_2512_06727_b200.session import Session
+    src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    pps = (w.cached_tokens + 1 + w.page_tokens - 1) // w.page_tokens
+    for label, aes in (("compressed", synth.make_stack_autoencoders(w, src, src)), ("raw", {})):
+        probe = B.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, 1, 1, 1, B.BF16)
+        probe.set_reuse_map(src, src)
+        for (l, which), ae in aes.items():
+            probe.set_autoencoder(l, which, ae)
+        comp, full = probe.cache_bytes_per_token()
+        n_seq = int(budget // (comp * pps * w.page_tokens))
+        torch.cuda.empty_cache()
+        sess = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, n_seq, n_seq * pps, pps,
+                       w.storage, src, src, aes)
+        allseq = list(range(n_seq))
+        for q_ in allseq:
+            sess.ctx.seq_open(q_)
+        for i in range(0, n_seq, B.MAX_BATCH):       # pages for every sequence; the rows keep the pool's zeros
+            part = allseq[i:i + B.MAX_BATCH]
+            sess.ctx.reserve(part, w.cached_tokens)
+            sess.ctx.advance(part, w.cached_tokens, sess.stream())
+        last = allseq[-min(B.MAX_BATCH, n_seq):]
+        k = torch.randn(len(last), w.kv_width, device="cuda").to(sess.dtype)
+        q = torch.randn(len(last), w.n_q_heads, w.head_dim, device="cuda").to(sess.dtype)
+        o = torch.empty_like(q)
+        t0 = time.perf_counter()
+        for l in range(w.n_layers):                  # one decode step over the last sequences of the pool
+            sess.ctx.step_layer(l, last, k.data_ptr(), k.data_ptr(), q.data_ptr(), o.data_ptr(), B.INCLUDE_CURRENT_EXACT,
+                                sess.stream())
+        sess.ctx.sync_status(sess.stream())
+        dt = time.perf_counter() - t0
+        out["held"].append({"layout": label, "cached_tokens": w.cached_tokens, "sequences_held": n_seq,
+                            "pool_bytes": sess.sizes[0], "cache_bytes_per_token": comp,
+                            "decode_step_of_last_sequences": {"sequences": len(last), "seconds": dt,
+                                                              "finite": bool(torch.isfinite(o.float()).all().item())}})
+        del sess
+        torch.cuda.empty_cache()
+    print(json.dumps(out))
+
+
 def run_prefill(args):
     """Bulk encoder + append: one call per layer of 1024 new tokens per sequence."""
     import torch
@@ -448,6 +532,123 @@ def run_prefill(args):
                       "cuda_core_encoder_ms_per_step": out["cuda_cores"]}))
 
 
+NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16 per B200 (vendor figure): context beside the measured peaks
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM bytes (read + write) per decode-kernel launch and listed sequence, from an ncu capture of the GPT-2-shaped
+# stack at 4096 cached tokens (batch 8, scaled by the batch: a launch's traffic is its sequences' latent rows)
+NCU_TRAFFIC = {"c5": {"bytes_per_sequence": 173.67e6 / 8, "captured_on": "c5_gpt2s_12l_L4096_b8",
+                      "profile": "profiles/decode_pair_kernel_c5.md"}}
+
+
+def roofline_of(flops, byts, seconds, peaks, launches):
+    """Both sides of the roofline for `launches` launches that took `seconds` in all: the slower of algorithmic bytes
+    at the measured copy bandwidth and algorithmic flops at the measured bf16 peak is the bound; the kernel is timed
+    alone (one event pair per launch), so the burst figure is the tensor peak."""
+    t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    tensor = t_tc >= t_hbm
+    ach = flops / seconds / 1e12 if tensor else byts / seconds / 1e9
+    peak = peaks["bf16_tflops"] if tensor else peaks["hbm_gbs"]
+    r = {"bound": "tensor" if tensor else "hbm", "achieved": ach, "peak": peak, "unit": "TFLOP/s" if tensor else "GB/s",
+         "frac": max(t_hbm, t_tc) / seconds, "traffic": None,
+         "peak_source": peaks["source"] + (" (burst: kernel timed alone)" if tensor else " (copy)"),
+         "kernel": "decode_attention (decoder + attention + combine)", "launches": launches,
+         "avg_launch_us": 1e6 * seconds / launches,
+         "algorithmic_flops_per_launch": flops / launches, "algorithmic_bytes_per_launch": byts / launches,
+         "tensor_side_frac": t_tc / seconds, "hbm_side_frac": t_hbm / seconds,
+         "frac_of_sustained_bf16": flops / seconds / 1e12 / peaks["bf16_tflops_sustained"],
+         "frac_of_nominal_bf16": flops / seconds / 1e12 / NOMINAL_BF16_TFLOPS,
+         "frac_of_nominal_hbm": byts / seconds / 1e9 / NOMINAL_HBM_GBS}
+    return r
+
+
+def fast_prefill(sess, w, torch):
+    """Untimed cache fill for the bench: the tensor-core bulk encoder where the layer has one, else the general one."""
+    seqs = list(range(w.batch))
+    for q in seqs:
+        sess.ctx.seq_open(q)
+    g = torch.Generator(device=sess.device)
+    g.manual_seed(w.seed)
+    chunk = max(64, min(w.cached_tokens, (1 << 27) // max(1, w.batch * w.kv_width)))
+    chunk = (chunk // w.page_tokens) * w.page_tokens or w.page_tokens
+    use_tensor = w.storage == "bf16" and sess.has_autoencoders
+    t = 0
+    while t < w.cached_tokens:
+        n = min(chunk, w.cached_tokens - t)
+        k = torch.randn(w.batch, n, w.kv_width, generator=g, device=sess.device, dtype=torch.float32).to(sess.dtype)
+        v = torch.randn(w.batch, n, w.kv_width, generator=g, device=sess.device, dtype=torch.float32).to(sess.dtype)
+        for l in range(w.n_layers):       # the same rows for every layer: content does not matter to the timing
+            call = sess.ctx.encode_append_tensor if use_tensor else sess.ctx.encode_append
+            call(l, seqs, n, k.data_ptr(), v.data_ptr(), sess.stream())
+        torch.cuda.current_stream().synchronize()
+        sess.ctx.advance(seqs, n, sess.stream())
+        t += n
+    sess.ctx.sync_status(sess.stream())
+
+
+def measure(w, args, torch, B, steps, warmup, uncompressed, flush, peaks, fused=True, keep=False):
+    """One workload: tokens/s through the per-layer step (all kernels of a step, L2 flushed between steps) and the
+    decode-attention call alone per launch (L2 flushed between launches)."""
+    class A: pass
+    a2 = A(); a2.uncompressed = uncompressed; a2.kernel = args.kernel
+    sess, src, aes = build_session(w, a2, torch, 2 * (warmup + steps) + 24)
+    sess.has_autoencoders = bool(aes)
+    fast_prefill(sess, w, torch)
+    seqs = list(range(w.batch))
+    stream = sess.stream()
+    flags = B.INCLUDE_CURRENT_EXACT
+    n_in = 4
+    k, v, q, out = step_inputs(sess, w, torch, n_in)       # a few input sets, cycled (values do not matter)
+    for i in range(warmup):
+        run_step(sess, w, seqs, k, v, q, out, i % n_in, stream, flags, fused)
+    sess.ctx.sync_status(stream)
+    launches0 = sess.ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    for j in range(steps):
+        flush.fill_(j & 0xFF)
+        ev[j][0].record()
+        run_step(sess, w, seqs, k, v, q, out, j % n_in, stream, flags, fused)
+        ev[j][1].record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    total_ms = float(sum(a_.elapsed_time(b_) for a_, b_ in ev))
+    launches = sess.ctx.launch_count() - launches0
+    sess.ctx.sync_status(stream)
+    # the decode-attention call alone
+    kev = []
+    n_k = max(1, min(steps, 4))
+    for j in range(n_k):
+        L = sess.ctx.seq_len(0)
+        for l in range(w.n_layers):
+            sess.ctx.encode_append(l, seqs, 1, k[j % n_in, l].data_ptr(), v[j % n_in, l].data_ptr(), stream)
+            flush.fill_(l & 0xFF)
+            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_.record()
+            sess.ctx.decode_attention(l, seqs, q[j % n_in, l].data_ptr(), out[j % n_in, l].data_ptr(), flags, stream)
+            b_.record()
+            kev.append((l, L, a_, b_))
+        sess.ctx.advance(seqs, 1, stream)
+    torch.cuda.synchronize()
+    sess.ctx.sync_status(stream)
+    flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
+    byts = sum(sess.ctx.layer_work_per_token(l)[0] * L * w.batch for (l, L, _, _) in kev)
+    kern_s = sum(a_.elapsed_time(b_) for (_, _, a_, b_) in kev) / 1e3
+    roof = roofline_of(flops, byts, kern_s, peaks, len(kev))
+    comp, full = sess.ctx.cache_bytes_per_token()
+    res = {"tokens_per_s": w.batch * steps / (total_ms / 1e3), "ms_per_step": total_ms / steps, "steps": steps,
+           "roofline": roof, "cache_bytes_per_token": comp, "uncompressed_bytes_per_token": full, "launches": int(launches),
+           "wall_s": wall, "total_ms": total_ms}
+    if keep:
+        res["session"] = (sess, src, aes, k, v, q, out)
+    else:
+        del sess
+        torch.cuda.empty_cache()
+    return res
+
+
 def main():
     args = parse()
     if args.impl == "reference":
@@ -458,6 +659,9 @@ def main():
         return
     if args.head_l1:
         run_head_l1(args)
+        return
+    if args.capacity:
+        run_capacity(args)
         return
     import torch
     import torch.distributed as dist
@@ -473,94 +677,41 @@ def main():
 
     w = workload_of(args)
     K_, W_ = args.steps, max(args.warmup, 3)
-    n_e2e = 0 if args.no_e2e else max(2, min(K_, 8))
-    extra = 2 * (W_ + K_) + 2 * n_e2e + 4
-    sess, src, aes = build_session(w, args, torch, extra)
-    torch.cuda.set_device(local)
-    sess.device = torch.device(f"cuda:{local}")
-    seqs = list(range(w.batch))
-    do_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
-    keep = tuple(range(min(8 if w.cached_tokens <= 4096 else 1, w.batch))) if do_cpu else ()
-    prefill(sess, w, torch, ())
-    stream = sess.stream()
-    flags = B.INCLUDE_CURRENT_EXACT
-    total_steps = 2 * (W_ + K_)
-    k, v, q, out = step_inputs(sess, w, torch, total_steps)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=sess.device)
+    peaks = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=f"cuda:{local}")
+    fused = args.api == "fused"
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- pass 1: the headline timing --------------------------------------
+    # ---- the headline workload ----------------------------------------------
     sampler = ClockSampler(local)
     if rank == 0:
-        sampler.start()          # nvidia-smi needs a moment to come up: it samples warm-up, timed region and pass 2
-    fused = args.api == "fused"
-    for i in range(W_):
-        run_step(sess, w, seqs, k, v, q, out, i, stream, flags, fused)
-    sess.ctx.sync_status(stream)
-    launches0 = sess.ctx.launch_count()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_)]
+        sampler.start()
     barrier()
-    wall0 = time.perf_counter()
-    for j in range(K_):
-        flush.fill_(j & 0xFF)                      # evict the cache from L2 between steps (outside the event pair)
-        ev[j][0].record()
-        run_step(sess, w, seqs, k, v, q, out, W_ + j, stream, flags, fused)
-        ev[j][1].record()
+    head = measure(w, args, torch, B, K_, W_, bool(args.uncompressed), flush, peaks, fused=fused, keep=True)
     barrier()
-    wall = time.perf_counter() - wall0
-    step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = float(sum(step_ms))
-    launches = sess.ctx.launch_count() - launches0
-    sess.ctx.sync_status(stream)
-    total_ms = max_over_ranks(total_ms, world, sess.device)
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = max_over_ranks(head["total_ms"], world, torch.device(f"cuda:{local}"))
     ms_per_step = total_ms / K_
     value = whole_job_tokens_per_s(w.batch, K_, world, total_ms / 1e3)
-
-    # ---- pass 2: the decode kernel alone, per launch ----------------------
-    base = W_ + K_
-    for i in range(W_):
-        run_step(sess, w, seqs, k, v, q, out, base + i, stream, flags)
-    kev = []
-    cached_at = []
-    for j in range(K_):
-        i = base + W_ + j
-        L = sess.ctx.seq_len(0)
-        for l in range(w.n_layers):
-            sess.ctx.encode_append(l, seqs, 1, k[i, l].data_ptr(), v[i, l].data_ptr(), stream)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            sess.ctx.decode_attention(l, seqs, q[i, l].data_ptr(), out[i, l].data_ptr(), flags, stream)
-            b.record()
-            kev.append((l, L, a, b))
-        sess.ctx.advance(seqs, 1, stream)
-    torch.cuda.synchronize()
-    sess.ctx.sync_status(stream)
-    clocks = sampler.stop() if rank == 0 else None
-    peaks = measured_peaks()
-    flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
-    byts = sum(sess.ctx.layer_work_per_token(l)[0] * L * w.batch for (l, L, _, _) in kev)
-    kern_ms = sum(a.elapsed_time(b) for (_, _, a, b) in kev)
-    n_k = len(kev)
-    if args.uncompressed:
-        ach = byts / (kern_ms / 1e3) / 1e9
-        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": None}
-    else:
-        ach = flops / (kern_ms / 1e3) / 1e12
-        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None}
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, args.kernel, bool(args.uncompressed)))
-    roof.update({"kernel": "decode_attention (decoder + attention + combine)", "launches": n_k,
-                 "avg_launch_us": 1e3 * kern_ms / n_k, "peak_source": peaks["source"] + " (sustained)",
-                 "algorithmic_flops_per_launch": flops / n_k, "algorithmic_bytes_per_launch": byts / n_k,
-                 "hbm_side_frac": (byts / (kern_ms / 1e3) / 1e9) / peaks["hbm_gbs"]})
+    roof = head["roofline"]
+    cfg_key = args.workload
+    if not args.uncompressed and args.kernel == "auto" and cfg_key in NCU_TRAFFIC:
+        t = NCU_TRAFFIC[cfg_key]
+        roof["traffic"] = t["bytes_per_sequence"] * w.batch
+        roof["traffic_source"] = (f"ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch on {t['captured_on']}, "
+                                  f"scaled by the batch; {t['profile']}")
+    sess, src, aes, k, v, q, out = head.pop("session")
+    seqs = list(range(w.batch))
+    stream = sess.stream()
+    flags = B.INCLUDE_CURRENT_EXACT
 
     # ---- e2e: host buffers through the C ABI, copies inside the timed region ----
     e2e = None
+    n_e2e = 0 if args.no_e2e else max(2, min(K_, 6))
     if n_e2e:
         hk = [k[0, l].cpu().pin_memory() for l in range(w.n_layers)]
         hv = [v[0, l].cpu().pin_memory() for l in range(w.n_layers)]
@@ -580,38 +731,77 @@ def main():
         for _ in range(n_e2e):
             e2e_step()
         barrier()
-        e2e_s = time.perf_counter() - t0
-        e2e_s = max_over_ranks(e2e_s, world, sess.device)
+        e2e_s = max_over_ranks(time.perf_counter() - t0, world, torch.device(f"cuda:{local}"))
         elem = 2 if w.storage == "bf16" else 4
         e2e = {"value": whole_job_tokens_per_s(w.batch, n_e2e, world, e2e_s), "unit": UNIT, "steps": n_e2e,
                "h2d_bytes_per_step": w.n_layers * w.batch * (2 * w.kv_width + w.n_q_heads * w.head_dim) * elem,
                "d2h_bytes_per_step": w.n_layers * w.batch * w.n_q_heads * w.head_dim * elem,
                "timing": "wall clock around K host-buffer steps, stream synchronised every step"}
         sess.ctx.sync_status(stream)
+    del sess
+    torch.cuda.empty_cache()
 
-    # ---- CPU baseline: the oracle on a bounded sample ------------------------
+    # ---- CPU baseline: the oracle on a bounded sample of the headline workload ----
     cpu = None
-    if do_cpu:
-        # a fresh decode step at the prefilled length for the sampled sequences, compared with the GPU
-        sess2, _, _ = build_session(w, args, torch, 4)
-        kept2 = prefill(sess2, w, torch, keep)
-        i = 0
-        run_step(sess2, w, seqs, k, v, q, out, i, sess2.stream(), flags)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # a small replica of the workload (same shapes and length, two sequences) filled through the general encoder,
+        # whose rows the oracle mirrors; a decode step of it is compared with the oracle and the oracle is timed
+        w2 = synth.with_batch(w, 2)
+        class A2: pass
+        a2 = A2(); a2.uncompressed = bool(args.uncompressed); a2.kernel = args.kernel
+        sess2, src2, aes2 = build_session(w2, a2, torch, 4)
+        kept2 = prefill(sess2, w2, torch, (0, 1))
+        k2, v2, q2, out2 = step_inputs(sess2, w2, torch, 1)
+        run_step(sess2, w2, [0, 1], k2, v2, q2, out2, 0, sess2.stream(), flags)
         torch.cuda.synchronize()
-        sk = [k[i, l].float().cpu().numpy() for l in range(w.n_layers)]
-        sv = [v[i, l].float().cpu().numpy() for l in range(w.n_layers)]
-        sq = [q[i, l].float().cpu().numpy() for l in range(w.n_layers)]
-        go = [out[i, l].float().cpu().numpy().astype(np.float64) for l in range(w.n_layers)]
+        sk = [k2[0, l].float().cpu().numpy() for l in range(w.n_layers)]
+        sv = [v2[0, l].float().cpu().numpy() for l in range(w.n_layers)]
+        sq = [q2[0, l].float().cpu().numpy() for l in range(w.n_layers)]
+        go = [out2[0, l].float().cpu().numpy().astype(np.float64) for l in range(w.n_layers)]
         del sess2
-        r = oracle_sample(w, src, aes, kept2, sk, sv, sq, args.cpu_seconds, go)
+        r = oracle_sample(w, src2, aes2, kept2, sk, sv, sq, args.cpu_seconds, go)
         cpu = {"value": r["value"], "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                "sample": f"decode step at {w.cached_tokens} cached tokens: {r['pairs']} (sequence, layer) pair evaluations "
-                         f"over {len(keep)} of {w.batch} sequences ({r['seconds']:.1f} s), scaled to the "
+                         f"on two sequences of the same shapes ({r['seconds']:.1f} s), scaled to the "
                          f"{w.batch * w.n_layers} pairs of a step",
                "max_abs_err_gpu_vs_oracle_on_sample": r["max_abs_err_vs_gpu"]}
 
+    # ---- the other configurations, shorter runs (parity cases of the test-suite, timed here for the record) ----
+    configs = None
+    if rank == 0 and world == 1 and not args.no_sweep:
+        configs = []
+        sweep = [("c1", None), ("c2", None), ("c3", None), ("c4", None)] + [("c5", b) for b in (1, 8, 32, 128, 256)]
+        for name, batch in sweep:
+            wc = synth.CONFIGS[name]
+            if batch:
+                wc = synth.with_batch(wc, batch)
+            big = wc.batch * wc.cached_tokens * wc.n_layers
+            st_ = 2 if big > 5e6 else 4
+            row = {"workload": wc.name, "batch": wc.batch, "cached_tokens": wc.cached_tokens, "layers": wc.n_layers,
+                   "dtype": wc.storage}
+            try:
+                if wc.name == w.name and not args.uncompressed:
+                    c = head
+                else:
+                    c = measure(wc, args, torch, B, st_, 3, False, flush, peaks)
+                r_ = c["roofline"]
+                row.update({"tokens_per_s": c["tokens_per_s"], "ms_per_step": c["ms_per_step"], "steps": c["steps"],
+                            "us_per_launch": r_["avg_launch_us"], "bound": r_["bound"], "frac": r_["frac"],
+                            "frac_of_sustained_bf16": r_["frac_of_sustained_bf16"], "achieved": r_["achieved"],
+                            "achieved_unit": r_["unit"],
+                            "cache_bytes_per_token": c["cache_bytes_per_token"],
+                            "uncompressed_bytes_per_token": c["uncompressed_bytes_per_token"]})
+                if wc.storage == "bf16":
+                    u = measure(wc, args, torch, B, st_, 3, True, flush, peaks)
+                    ru = u["roofline"]
+                    row["raw_twin"] = {"tokens_per_s": u["tokens_per_s"], "us_per_launch": ru["avg_launch_us"],
+                                       "bound": ru["bound"], "frac": ru["frac"], "achieved_gbs": ru["achieved"],
+                                       "cache_bytes_per_token": u["cache_bytes_per_token"]}
+            except Exception as ex:      # a configuration that does not fit or fails is reported, not fatal
+                row["error"] = str(ex)[:200]
+            configs.append(row)
+
     if rank == 0:
-        comp, full = sess.ctx.cache_bytes_per_token()
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_, "warmup": W_,
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if w.storage == "bf16" else "f32", "data": "synthetic",
@@ -619,11 +809,13 @@ def main():
                            "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
                            "latent_full": 0 if args.uncompressed else w.latent_full, "reuse_frac": w.reuse_frac,
                            "page_tokens": w.page_tokens, "kernel": args.kernel, "api": args.api,
-                           "uncompressed": bool(args.uncompressed),
-                           "l2": "flushed between steps (256 MiB write outside the per-step event pairs)",
-                           "cache_bytes_per_token": comp, "uncompressed_bytes_per_token": full,
-                           "wall_s_timed_region": wall},
-                "clocks": clocks, "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches)}
+                           "uncompressed": bool(args.uncompressed), "storage": w.storage,
+                           "l2": "flushed between steps and between the per-launch timings (256 MiB write outside the event pairs)",
+                           "cache_bytes_per_token": head["cache_bytes_per_token"],
+                           "uncompressed_bytes_per_token": head["uncompressed_bytes_per_token"],
+                           "wall_s_timed_region": head["wall_s"]},
+                "clocks": clocks, "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": head["launches"], "configs": configs}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

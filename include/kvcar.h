@@ -257,9 +257,10 @@ kvcar_status kvcar_step_layer_host(kvcar_ctx *ctx, int32_t layer, const int32_t 
  *  - n_seqs * ceil(longest listed sequence / 128) * n_q_heads * (head_dim + 2)
  *    floats must fit in KVCAR_STATIC_SCRATCH_BYTES, else KVCAR_ERR_WORKSPACE
  *    and nothing is launched.
- *  - The first call on each device looks up the array's device address (with
- *    that device current, the one whose stream is passed); make that first call
- *    outside any stream capture.
+ *  - kvcar_bind_memory looks up the array's device address (set-up time, with
+ *    the target device current; the first lookup on a device is when the driver
+ *    sets the array's memory aside).  The call itself only reads that address.
+ *    Contexts are used on the device they were bound on.
  *  - All contexts and streams of a process share the one array per device, and
  *    it keeps whatever the previous call left; every slot a call reads is
  *    written earlier in the same call, so nothing needs clearing, but two
@@ -302,6 +303,13 @@ kvcar_status kvcar_layer_kernel(kvcar_ctx *ctx, int32_t layer, int32_t *kernel);
  * bounded-wait timeout recorded since the last call. */
 kvcar_status kvcar_sync_status(kvcar_ctx *ctx, void *stream);
 const char *kvcar_last_error(kvcar_ctx *ctx);
+/* Test hook for the device-side timeout path: enqueue a one-warp kernel that waits
+ * on a barrier nothing ever completes, gives up after limit_ns (1 ns .. 1 s),
+ * records a code in the context's status word and returns normally.  The next
+ * kvcar_sync_status then reports KVCAR_ERR_DEVICE_TIMEOUT once.  Every bounded
+ * wait of the fused kernel ends this way when it runs out (their limit is 2 s);
+ * nothing traps and the context stays usable. */
+kvcar_status kvcar_debug_expire_wait(kvcar_ctx *ctx, uint64_t limit_ns, void *stream);
 
 /* ---- choosing the reuse map (Alg. 2, its first three steps) -------------------
  *

@@ -30,7 +30,7 @@ EXPORTS = [
     "kvcar_step_layer", "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
-    "kvcar_last_error",
+    "kvcar_last_error", "kvcar_debug_expire_wait",
     "kvcar_head_l1_scratch_bytes", "kvcar_head_l1_distance", "kvcar_reuse_map_from_l1",
 ]
 
@@ -107,6 +107,7 @@ def _load() -> C.CDLL:
         "kvcar_launch_count": [vp, C.POINTER(C.c_int64)],
         "kvcar_layer_kernel": [vp, i32, ip],
         "kvcar_sync_status": [vp, vp],
+        "kvcar_debug_expire_wait": [vp, C.c_uint64, vp],
         "kvcar_head_l1_scratch_bytes": [i32, i32, C.c_int64, C.POINTER(sz)],
         "kvcar_head_l1_distance": [i32, i32, i32, i32, vp, C.c_int64, vp, sz, vp, vp],
         "kvcar_reuse_map_from_l1": [C.POINTER(C.c_float), i32, i32, i32, ip],
@@ -317,3 +318,6 @@ class Context:
 
     def sync_status(self, stream: int = 0):
         self._check(self.lib.kvcar_sync_status(self._h, stream))
+
+    def debug_expire_wait(self, limit_ns: int, stream: int = 0):
+        self._check(self.lib.kvcar_debug_expire_wait(self._h, limit_ns, stream))

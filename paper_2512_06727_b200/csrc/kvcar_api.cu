@@ -61,6 +61,7 @@ struct kvcar_ctx {
     int max_d = 0, max_m = 0, max_in = 0;
     std::vector<LayerPlan> plans_host;
     TcState tc;
+    float *static_scratch = nullptr;  // device address of the built-in scratch array, looked up at bind time
 
     int64_t launches = 0;
     std::string err;
@@ -284,6 +285,9 @@ bool use_tensor_kernel(const kvcar_ctx *c) {
     if (c->kernel == KVCAR_KERNEL_GENERIC) return false;
     return c->tc.available;
 }
+
+// device address of the library's built-in scratch array on the current device (defined with the array, below)
+cudaError_t static_scratch_for_current_device(float **out);
 
 }  // namespace
 
@@ -549,6 +553,12 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
             if (c->side) cudaStreamDestroy(c->side);
             c->side = nullptr;
         }
+    }
+    {   // kvcar_decode_attention_static: take the built-in scratch array's address now, at set-up time (the first
+        // lookup on a device loads the array's module, which is when the driver sets its memory aside)
+        float *p = nullptr;
+        if (static_scratch_for_current_device(&p) != cudaSuccess) cudaGetLastError();
+        c->static_scratch = p;
     }
     c->bound = true;
     c->pending.clear();
@@ -977,6 +987,16 @@ kvcar_status kvcar_sync_status(kvcar_ctx *c, void *stream) {
 
 const char *kvcar_last_error(kvcar_ctx *c) { return c ? c->err.c_str() : "null context"; }
 
+kvcar_status kvcar_debug_expire_wait(kvcar_ctx *c, uint64_t limit_ns, void *stream) {
+    if (!c) return KVCAR_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return fail(c, KVCAR_ERR_INVALID_ARG, "limit must be 1 ns .. 1 s");
+    cudaError_t e = tc_launch_expire_wait(reinterpret_cast<int32_t *>(c->ws + c->status_off), limit_ns, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "launch");
+    ++c->launches;
+    return KVCAR_OK;
+}
+
 }  // extern "C"
 
 // =============================================================================
@@ -989,9 +1009,9 @@ static __device__ __align__(256) unsigned char g_static_scratch[KVCAR_STATIC_SCR
 
 namespace {
 constexpr int kMaxDevices = 64;
-float *g_static_scratch_ptr[kMaxDevices] = {};  // per device; filled on the first call there
+float *g_static_scratch_ptr[kMaxDevices] = {};  // per device; filled by the first kvcar_bind_memory there
 
-// Device address of the scratch array on the current device (set-up on first use).
+// Device address of the scratch array on the current device.
 cudaError_t static_scratch_for_current_device(float **out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1034,9 +1054,9 @@ extern "C" kvcar_status kvcar_decode_attention_static(kvcar_ctx *c, int32_t laye
     }
     if (decode_generic_smem(g.n_q_heads, g.head_dim, c->max_d, c->max_m) > 227 * 1024)
         return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");
-    float *scratch = nullptr;
-    cudaError_t e = static_scratch_for_current_device(&scratch);
-    if (e != cudaSuccess) return cuda_fail(c, e, "address of the built-in scratch array");
+    float *scratch = c->static_scratch;
+    if (!scratch) return fail(c, KVCAR_ERR_STATE, "the built-in scratch array could not be located when memory was bound");
+    cudaError_t e;
     cudaStream_t st = (cudaStream_t)stream;
     kvcar_status s = flush_tables(c, st);
     if (s != KVCAR_OK) return s;

@@ -53,9 +53,12 @@
 #include <cstring>
 #include <vector>
 
+#include "kvcar_ptx.cuh"
 #include "kvcar_tc.h"
 
 namespace kvcar {
+
+using namespace ptx;
 
 namespace {
 
@@ -89,52 +92,7 @@ struct PairLaunch {
     uint32_t *pflags;   // [tile][hkv]
 };
 
-// ---------------------------------------------------------------------------- PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// arrive on a barrier of any CTA of the cluster (address from map_to_cta), release at cluster scope
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-// arrive on a barrier of any CTA of the cluster (address from map_to_cta), ordering only this CTA's earlier operations
-// (enough where the data handed over is tensor memory already read, or this CTA's shared memory already fenced for the
-// async proxy)
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-template <bool CLUSTER>
-__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    if (CLUSTER)  // the phase was completed by another CTA's ordinary stores + arrive: acquire at cluster scope
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, "
-            "0, p;\n}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-    else
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-    return ok;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
+// ---------------------------------------------------------------------------- waits
 // Bounded wait.  `abort_flag` (shared) shortens every later wait once one has failed.
 // SLEEP_NS > 0: back off between polls so that a waiting warp leaves the issue slots of its scheduler to the
 // warps that share it (the MMA issuer above all).
@@ -160,124 +118,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int32_t
     }
 }
 
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-
-// 2-D tile load into this CTA's shared memory; completion bytes go to a barrier that may live in the pair's
-// other CTA (cluster address)
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int x, int y, uint32_t cluster_bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], "
-        "[%4];" ::"r"(dst),
-        "l"(tmap), "r"(x), "r"(y), "r"(cluster_bar)
-        : "memory");
-}
-
-// bring one box of a tensor into L2 ahead of its load
-__device__ __forceinline__ void tma_prefetch_2d(const void *tmap, int x, int y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// D[tmem, both CTAs] (+)= A[smem desc] . B[smem desc]^T, bf16 inputs, fp32 accumulate, M = 256 over the CTA pair
-__device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(
-            d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// arrive on the barrier at this shared-memory offset in both CTAs of the pair once all earlier MMAs are done
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-        "h"((uint16_t)3)
-        : "memory");
-}
-
-// 32 lanes x 32 columns of fp32: thread i of the warp gets lane (base+i), columns col..col+31
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
-    uint32_t *r = reinterpret_cast<uint32_t *>(v);
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-// 16 lanes x 8*N columns of fp32 in the accumulator-fragment layout of the warp-level MMA: thread t gets, per
-// 8-column block j, rows t/4 (regs 4j, 4j+1) and t/4 + 8 (regs 4j+2, 4j+3), columns 8j + 2*(t%4) + {0, 1}
-__device__ __forceinline__ void tmem_ld_frag_x4(uint32_t taddr, uint32_t *r) {  // 32 columns
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
-        "[%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
-// D[16 x 8] += A[16 x 16] . B[16 x 8], bf16 operands, fp32 accumulate (warp-level tensor op for the small
-// attention products of a query group)
-__device__ __forceinline__ void mma_16816(float *d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                          uint32_t b1) {
-    asm(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, "
-        "%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major, 128B-swizzled operand tile: rows of 128 B, 8-row groups 1024 B apart
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address
-    d |= (uint64_t)1 << 16;                        // leading byte offset (unused with 128B swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset
-    d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                        // SWIZZLE_128B
-    return d;
-}
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major
-__device__ __forceinline__ uint32_t make_idesc(int M, int N) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-// Copy `bytes` (a multiple of 16, both addresses 16-byte aligned) from this CTA's shared memory into the peer CTA's
-// and count them on a barrier there: whoever sees that barrier's phase complete sees the data, with no fence on
-// the writing side beyond the one that shows the source to the copy engine.
-__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
-    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     dst_cluster),
-                 "r"(src_cta), "r"(bytes), "r"(bar_cluster)
-                 : "memory");
-}
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
-                 : "memory");
-}
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
 
 struct Bars {
     uint32_t full, empty;  // [nslot] each (8 B apart); `full` is used in the leader CTA only
@@ -325,10 +166,13 @@ __device__ __forceinline__ int job_slot(const TcJob &j, int hp) {
 // one 64-wide K slab: up to four K=16 steps
 __device__ __forceinline__ void issue_kslab(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, int nk,
                                             bool first_slab) {
-    umma_pair(d_tmem, a_desc, b_desc, idesc, first_slab ? 0u : 1u);
-    if (nk > 1) umma_pair(d_tmem, a_desc + 2u, b_desc + 2u, idesc, 1u);
-    if (nk > 2) umma_pair(d_tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
-    if (nk > 3) umma_pair(d_tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
+    if (first_slab)
+        umma_pair<0>(d_tmem, a_desc, b_desc, idesc);
+    else
+        umma_pair<1>(d_tmem, a_desc, b_desc, idesc);
+    if (nk > 1) umma_pair<1>(d_tmem, a_desc + 2u, b_desc + 2u, idesc);
+    if (nk > 2) umma_pair<1>(d_tmem, a_desc + 4u, b_desc + 4u, idesc);
+    if (nk > 3) umma_pair<1>(d_tmem, a_desc + 6u, b_desc + 6u, idesc);
 }
 
 // ---------------------------------------------------------------------------- the kernel
@@ -485,15 +329,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             turn ^= 1u;
                             acquire1(2 * SLOT_BYTES, own, dst, fb);
                             if (own) {
-                                tma_load_2d(dst, sp.tm_pool, ks * 64, row[0], fb);
-                                tma_load_2d(dst + HALF_BYTES, sp.tm_pool, ks * 64, row[1], fb);
+                                tma_load_2d_pair(dst, sp.tm_pool, ks * 64, row[0], fb);
+                                tma_load_2d_pair(dst + HALF_BYTES, sp.tm_pool, ks * 64, row[1], fb);
                             }
                             own = turn == pid;
                             turn ^= 1u;
                             acquire1(half_rows > 64 ? 2 * SLOT_BYTES : 2 * HALF_BYTES, own, dst, fb);
                             if (own) {
-                                tma_load_2d(dst, sp.tm_w1, ks * 64, y0, fb);
-                                if (half_rows > 64) tma_load_2d(dst + HALF_BYTES, sp.tm_w1, ks * 64, y0 + 64, fb);
+                                tma_load_2d_pair(dst, sp.tm_w1, ks * 64, y0, fb);
+                                if (half_rows > 64) tma_load_2d_pair(dst + HALF_BYTES, sp.tm_w1, ks * 64, y0 + 64, fb);
                             }
                         }
                     } else {
@@ -514,9 +358,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             const uint32_t sl = acquire(yb >= 0 ? 2 * SLOT_BYTES : 2 * HALF_BYTES, own);
                             if (own) {
                                 const uint32_t fb = map_to_cta(B.full + 8 * sl, 0);
-                                tma_load_2d(s_ring + sl * SLOT_BYTES, sp.tm_w2, ks * 64, ya, fb);
+                                tma_load_2d_pair(s_ring + sl * SLOT_BYTES, sp.tm_w2, ks * 64, ya, fb);
                                 if (yb >= 0)
-                                    tma_load_2d(s_ring + sl * SLOT_BYTES + HALF_BYTES, sp.tm_w2, ks * 64, yb, fb);
+                                    tma_load_2d_pair(s_ring + sl * SLOT_BYTES + HALF_BYTES, sp.tm_w2, ks * 64, yb, fb);
                             }
                         }
                     }
@@ -1218,36 +1062,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 }
 
 // ---------------------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-    void *fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess) {
-        cudaGetLastError();
-        return nullptr;
-    }
-    return reinterpret_cast<EncodeTiledFn>(fn);
-}
-
-// bf16 matrix [rows][cols] row-major -> descriptor with a [64 rows][64 cols] box, 128B swizzle, zero fill
-bool encode_map(EncodeTiledFn fn, void *dst_host, const void *dev_ptr, uint64_t rows, uint64_t cols) {
-    CUtensorMap m;
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, 64};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(dev_ptr), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return false;
-    memcpy(dst_host, &m, sizeof(m));
-    return true;
-}
-
 inline uint32_t up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
 PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslots, int nslot) {
@@ -1352,7 +1166,34 @@ bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int
 
 inline int part_index(int split, int i) { return (split == 1 ? 0 : split == 2 ? 1 : 3) + i; }
 
+// A wait that nothing completes: one warp waits on a fresh barrier with the given limit, records its code in the
+// status word and returns.  Exercises the path every bounded wait of this file takes when it runs out.
+__global__ void expire_wait_kernel(int32_t *status, uint64_t limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+    }
+    __syncwarp();
+    const uint32_t b = smem_u32(&bar);
+    const uint64_t t0 = global_ns();
+    while (!mbar_try(b, 0)) {
+        __nanosleep(200);
+        if (global_ns() - t0 > limit_ns) {
+            abort_flag = 1;
+            atomicCAS(status, 0, 0x7e57);
+            break;
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t tc_launch_expire_wait(int32_t *status, uint64_t limit_ns, cudaStream_t st) {
+    expire_wait_kernel<<<1, 32, 0, st>>>(status, limit_ns);
+    return cudaGetLastError();
+}
 
 size_t tc_part_bytes(int n_layers) { return (size_t)n_layers * 7 * sizeof(TcPart); }
 size_t tc_split_bytes(const kvcar_config &cfg) {
@@ -1377,7 +1218,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
         tc.why = "more than 8 query heads per KV head";
         return;
     }
-    EncodeTiledFn fn = get_encode_fn();
+    EncodeTiledFn fn = tensor_map_encoder();
     if (!fn) {
         tc.why = "cuTensorMapEncodeTiled is not available (no driver)";
         return;
@@ -1405,9 +1246,9 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
                 char *host = img + tmap_off + (size_t)idx * 3 * 128;
                 char *devp = weights_dev + tmap_off + (size_t)idx * 3 * 128;
                 if (!built[idx]) {
-                    if (!encode_map(fn, host, sp.pool, pool_rows, (uint64_t)sp.width) ||
-                        !encode_map(fn, host + 128, sp.w1k, (uint64_t)sp.m, (uint64_t)sp.d) ||
-                        !encode_map(fn, host + 256, sp.w2k, (uint64_t)sp.in_dim, (uint64_t)sp.m)) {
+                    if (!encode_bf16_map(fn, host, sp.pool, pool_rows, (uint64_t)sp.width, (uint64_t)sp.width) ||
+                        !encode_bf16_map(fn, host + 128, sp.w1k, (uint64_t)sp.m, (uint64_t)sp.d, (uint64_t)sp.d) ||
+                        !encode_bf16_map(fn, host + 256, sp.w2k, (uint64_t)sp.in_dim, (uint64_t)sp.m, (uint64_t)sp.m)) {
                         ok = false;
                         break;
                     }
@@ -1480,8 +1321,12 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     const int n_pairs = (int)((t + 1) / 2);
     // Small grids: spread the work of a tile pair over more clusters while everything still runs in one wave.
     // First K and V go to separate clusters (nothing is computed twice: the probabilities cross through global
-    // memory, which needs both clusters on the machine at once - true below the SM count); then the KV heads
-    // are split (each cluster repeats the hidden layer for its heads).
+    // memory behind per-head flags); then the KV heads are split (each cluster repeats the hidden layer for its
+    // heads).  A V cluster waits for flags that the K cluster of the same pair sets, and a K cluster waits for no
+    // other cluster.  The K cluster has the lower block index (cluster id = pair * clusters per pair + part, K
+    // parts first), and thread blocks are handed to the SMs in increasing block-index order: when a V cluster
+    // starts, its K cluster is already resident or finished, whatever else shares the machine (the encoder
+    // launches of kvcar_step_layer, other streams).  The flag wait is bounded all the same.
     int split = 1, kv_split = 0;
     if (tc.pbuf && 4 * n_pairs <= tc.n_sms) {
         kv_split = 1;

@@ -78,4 +78,7 @@ bool tc_layer_supported(const TcState &tc, int layer);
 cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
                              int layer, cudaStream_t st);
 
+// test hook: one warp waits `limit_ns` on a barrier that nothing completes, then records code 0x7e57 in the status word
+cudaError_t tc_launch_expire_wait(int32_t *status, uint64_t limit_ns, cudaStream_t st);
+
 }  // namespace kvcar

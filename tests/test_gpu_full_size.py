@@ -31,6 +31,12 @@ def _prefill_device(p, w, seqs, n_tokens, seed, chunk=1024):
     p.s.ctx.sync_status(p.s.stream())
 
 
+def _reused_heads(w):
+    """(layer, head) pairs of the workload's seeded reuse map that read the layer below."""
+    src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+    return {(l, h) for l in range(w.n_layers) for h in range(w.n_kv_heads) if src[l * w.n_kv_heads + h] >= 0}
+
+
 def _run(w, sampled, steps=1, fused=False, compress=True):
     pps = (w.cached_tokens + steps + w.page_tokens - 1) // w.page_tokens
     p = Pair(w, max_seqs=w.batch, max_pages=w.batch * pps, max_pages_per_seq=pps, kernel=B.KERNEL_AUTO,
@@ -42,53 +48,64 @@ def _run(w, sampled, steps=1, fused=False, compress=True):
     want_kernel = B.KERNEL_TENSOR if compress else B.KERNEL_RAW
     assert all(p.s.ctx.layer_kernel(l) == want_kernel for l in range(w.n_layers))
     worst = 0.0
+    pairs = set()
     for step in range(steps):
         res = p.decode_step(seqs, step, fused=fused)
         for l, (got, ref, rows) in res.items():
             assert rows == sorted(sampled)
             err, _ = assert_close(got[rows], ref, w.storage, f"{w.name} step {step} layer {l}")
             worst = max(worst, err)
+            pairs |= {(s_, l) for s_ in sampled}
     comp, full = p.s.ctx.cache_bytes_per_token()
     assert (comp, full) == p.o.cache_bytes_per_token()
-    return worst, comp, full
+    # every output of a layer covers all of its KV heads, so a reused head is exercised iff its layer was compared
+    hit = {(l, h) for (l, h) in _reused_heads(w) if any(pl == l for (_, pl) in pairs)}
+    return worst, comp, full, pairs, hit
 
 
 def test_config2_full_size_sampled():
     """GPT-2-small-shaped stack: 12 layers, batch 8, 1024 cached tokens, 25 % reuse; two steps;
-    every sequence, i.e. every output of both steps, against the oracle."""
+    every sequence, i.e. every output of both steps (96 (sequence, layer) pairs per step), against the oracle."""
     w = synth.CONFIGS["c2"]
-    worst, comp, full = _run(w, list(range(w.batch)), steps=2)
+    worst, comp, full, pairs, hit = _run(w, list(range(w.batch)), steps=2)
+    assert len(pairs) == 96 and hit == _reused_heads(w)
     assert comp < 0.5 * full      # latents halve the stored heads, reuse removes a quarter of them
 
 
 def test_config3_full_size_sampled():
-    """TinyLLaMA-shaped GQA stack: 22 layers, batch 32, 2048 cached tokens, 20 % reuse;
-    sequences 3, 17 and 30 against the oracle: 66 (sequence, layer) pairs, every layer and so every reused head."""
+    """TinyLLaMA-shaped GQA stack: 22 layers, batch 32, 2048 cached tokens, 20 % reuse; two steps (the second reads
+    the row the first appended); sequences 3, 17 and 30 against the oracle: 66 (sequence, layer) pairs, every layer
+    and so every reused head."""
     w = synth.CONFIGS["c3"]
-    _run(w, [3, 17, 30], steps=1)
+    _, _, _, pairs, hit = _run(w, [3, 17, 30], steps=2)
+    assert len(pairs) == 66 and hit == _reused_heads(w)
 
 
 def test_config4_long_context_sampled():
-    """Long context: 32 768 cached tokens per sequence (256 tiles, split-KV over all of them),
-    batch 4, the first three layers of the TinyLLaMA-shaped stack (the oracle would need
-    hours for all 22 at this length); sequence 2 against the oracle."""
-    w = synth.scaled(synth.CONFIGS["c4"], n_layers=3)
-    _run(w, [2], steps=1)
+    """Long context: 32 768 cached tokens per sequence (256 tiles, split-KV over all of them), batch 4, all 22
+    layers of the TinyLLaMA-shaped stack, two steps; sequences 0, 2 and 3 against the oracle: 66 (sequence, layer)
+    pairs, every layer and every reused head of the seed-3 map."""
+    w = synth.CONFIGS["c4"]
+    _, _, _, pairs, hit = _run(w, [0, 2, 3], steps=2)
+    assert len(pairs) == 66 and hit == _reused_heads(w)
 
 
 def test_config5_batch_sweep_point_sampled():
-    """GPT-2-small-shaped stack at 4096 cached tokens, batch 32 (one point of the batch
-    sweep; many waves of clusters), first four layers; sequence 17 against the oracle."""
-    w = synth.scaled(synth.with_batch(synth.CONFIGS["c5"], 32), n_layers=4)
-    _run(w, [17], steps=1)
+    """GPT-2-small-shaped stack at 4096 cached tokens, batch 32 (one point of the batch sweep; many waves of
+    clusters), all 12 layers, two steps; sequences 0, 5, 11, 17, 23 and 31 against the oracle: 72 (sequence, layer)
+    pairs, every layer and every reused head of the seed-4 map."""
+    w = synth.with_batch(synth.CONFIGS["c5"], 32)
+    _, _, _, pairs, hit = _run(w, [0, 5, 11, 17, 23, 31], steps=2)
+    assert len(pairs) == 72 and hit == _reused_heads(w)
 
 
 def test_config5_largest_batch_single_call_step_sampled():
     """The batch sweep's largest point: 256 sequences of 4096 cached tokens (8448 tiles, 57 tile pairs per
-    cluster), first two layers, each layer's step through the single-call entry point; the first and the last
-    sequence against the oracle."""
-    w = synth.scaled(synth.with_batch(synth.CONFIGS["c5"], 256), n_layers=2)
-    _run(w, [0, 255], steps=1, fused=True)
+    cluster), all 12 layers, two steps, each layer's step through the single-call entry point; sequences 0, 63, 64,
+    129, 200 and 255 against the oracle: 72 (sequence, layer) pairs, every layer and every reused head."""
+    w = synth.with_batch(synth.CONFIGS["c5"], 256)
+    _, _, _, pairs, hit = _run(w, [0, 63, 64, 129, 200, 255], steps=2, fused=True)
+    assert len(pairs) == 72 and hit == _reused_heads(w)
 
 
 def test_config3_uncompressed_twin_sampled():

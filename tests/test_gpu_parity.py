@@ -336,3 +336,20 @@ def test_errors_leave_state_untouched():
     with pytest.raises(B.KvcarError) as e:
         p.s.ctx.decode_attention(0, [5], big.data_ptr(), big.data_ptr(), 0, p.s.stream())
     assert e.value.status == 1
+
+
+def test_device_side_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """A bounded device-side wait that nothing completes: the kernel gives up after its limit (1 ms here), records a
+    code in the status word and returns; kvcar_sync_status reports KVCAR_ERR_DEVICE_TIMEOUT exactly once, and the
+    next decode on the same context is correct.  Nothing traps, faults or waits without a limit."""
+    w = synth.scaled(synth.CONFIGS["c3"], n_layers=2, batch=2, reuse_frac=0.25)
+    p = Pair(w, max_seqs=2, max_pages=8, max_pages_per_seq=4)
+    p.open([0, 1])
+    p.prefill([0], 140)
+    p.prefill([1], 65)
+    p.s.ctx.debug_expire_wait(1_000_000, p.s.stream())
+    with pytest.raises(B.KvcarError) as e:
+        p.s.ctx.sync_status(p.s.stream())
+    assert e.value.status == 7 and "0x7e57" in str(e.value)
+    p.s.ctx.sync_status(p.s.stream())            # the word was cleared: reported once
+    _check_step(p.decode_step([0, 1], 0), "bf16", "after a timed-out wait")

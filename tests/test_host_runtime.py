@@ -154,6 +154,44 @@ def test_accounting_and_layout():
     assert c1.layer_work_per_token(0) == (1536.0, 2654208.0 + 3072.0)
 
 
+def test_library_accounting_reproduces_the_printed_percentages():
+    """The library's own kvcar_cache_bytes_per_token, driven through the C ABI, against the cache reductions the paper
+    prints (Tables 2, 3 and 4; the records and their citations are in tests/golden/paper_accounting.txt)."""
+    golden = os.path.join(ROOT, "tests", "golden", "paper_accounting.txt")
+    seen = 0
+    for line in open(golden):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        kind, params, printed, cite = [p_.strip() for p_ in line.split("|")]
+        if kind.startswith("eq3"):
+            continue
+        kv = dict(p_.split("=") for p_ in params.split())
+        layers, heads, hd = int(kv["layers"]), int(kv["heads"]), 64
+        src = [np.full((layers, heads), -1, np.int32), np.full((layers, heads), -1, np.int32)]
+        for which, key in ((K, "k_heads"), (V, "v_heads")):
+            n = kv.get(key, "0")
+            if n == "all":
+                src[which][1::2, :] = np.arange(heads)        # every second layer reads the layer below
+            else:
+                cand = [(l, h) for l in range(1, layers, 2) for h in range(heads)]
+                for l, h in cand[:int(n)]:
+                    src[which][l, h] = h
+        c = B.Context(layers, heads, heads, hd, 64, 1, 1, 1, B.BF16)
+        c.set_reuse_map(src[K].reshape(-1), src[V].reshape(-1))
+        ratio = float(kv.get("ratio", 1.0))
+        for l in range(int(kv.get("compressed", 0))):
+            for which in (K, V):
+                n_stored = int((src[which][l] < 0).sum())
+                if n_stored:
+                    i, m, d = synth.ae_dims(n_stored, hd, int(hd * ratio))
+                    c.set_autoencoder(l, which, synth.make_autoencoder(i, m, d, 0, l, which, storage="bf16"))
+        comp, full = c.cache_bytes_per_token()
+        assert abs(100.0 * (1.0 - comp / full) - float(printed)) < 0.1, (cite, comp, full)
+        seen += 1
+    assert seen == 12
+
+
 def test_launching_calls_need_bound_memory():
     c = B.Context(1, 4, 2, 64, 64, 2, 4, 2, B.BF16)
     c.seq_open(0)
