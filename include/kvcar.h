@@ -79,6 +79,11 @@ typedef struct {
     int32_t max_pages;         /* physical pages shared by all sequences (and all layers)       */
     int32_t max_pages_per_seq; /* longest sequence = max_pages_per_seq * page_tokens tokens     */
     int32_t storage;           /* kvcar_dtype of q/k/v/out and of cache rows                    */
+    int32_t latent_quant;      /* 0: latent rows in the storage type.  1: int8 latent rows (Sec.
+                                  "Quantization", Eq. 4), one scale and one zero-point (fp32 each)
+                                  per cached row, kept beside the codes; needs bf16 storage, an
+                                  autoencoder on every (layer, K/V) that stores heads, and latent
+                                  widths that are multiples of 16                                */
 } kvcar_config;
 
 /*
@@ -285,6 +290,10 @@ kvcar_status kvcar_seq_len(kvcar_ctx *ctx, int32_t seq, int32_t *len);
  * row 0, bytes between rows, and elements per row (0 if the layer stores none). */
 kvcar_status kvcar_pool_layout(kvcar_ctx *ctx, int32_t layer, int32_t which, size_t *offset, size_t *row_pitch,
                                int32_t *width);
+/* int8 latent rows (config.latent_quant): byte offset, inside the pool buffer, of the layer's
+ * [max_pages*page_tokens][2] fp32 array of (scale, zero-point) per cached row; the codes are at
+ * kvcar_pool_layout's offset with a row pitch of `width` bytes.  Row r holds x ~ (code - zero-point) / scale. */
+kvcar_status kvcar_pool_quant_layout(kvcar_ctx *ctx, int32_t layer, int32_t which, size_t *param_offset);
 /* Bytes one cached token occupies over all layers: as configured, and with
  * neither autoencoders nor reuse (Eq. 3 per token and sequence). */
 kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *ctx, double *compressed, double *uncompressed);

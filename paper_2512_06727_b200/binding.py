@@ -28,7 +28,7 @@ EXPORTS = [
     "kvcar_bind_memory", "kvcar_set_kernel", "kvcar_seq_open", "kvcar_seq_close", "kvcar_reserve",
     "kvcar_encode_append", "kvcar_encode_append_tensor", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
     "kvcar_step_layer", "kvcar_step_layer_host",
-    "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout",
+    "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout", "kvcar_pool_quant_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
     "kvcar_last_error", "kvcar_debug_expire_wait",
     "kvcar_head_l1_scratch_bytes", "kvcar_head_l1_distance", "kvcar_reuse_map_from_l1",
@@ -43,7 +43,8 @@ class KvcarError(RuntimeError):
 
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "page_tokens",
-                                          "max_seqs", "max_pages", "max_pages_per_seq", "storage")]
+                                          "max_seqs", "max_pages", "max_pages_per_seq", "storage",
+                                          "latent_quant")]
 
 
 _FP = C.POINTER(C.c_float)
@@ -102,6 +103,7 @@ def _load() -> C.CDLL:
         "kvcar_debug_locate": [vp, i32, i32, ip, C.POINTER(C.c_int64)],
         "kvcar_seq_len": [vp, i32, ip],
         "kvcar_pool_layout": [vp, i32, i32, C.POINTER(sz), C.POINTER(sz), ip],
+        "kvcar_pool_quant_layout": [vp, i32, i32, C.POINTER(sz)],
         "kvcar_cache_bytes_per_token": [vp, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "kvcar_layer_work_per_token": [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "kvcar_launch_count": [vp, C.POINTER(C.c_int64)],
@@ -158,10 +160,10 @@ class Context:
     device addresses (ints, e.g. tensor.data_ptr()) for device buffers."""
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, page_tokens: int,
-                 max_seqs: int, max_pages: int, max_pages_per_seq: int, storage: int):
+                 max_seqs: int, max_pages: int, max_pages_per_seq: int, storage: int, latent_quant: int = 0):
         self.lib = load()
         self.cfg = Config(n_layers, n_q_heads, n_kv_heads, head_dim, page_tokens, max_seqs, max_pages,
-                          max_pages_per_seq, storage)
+                          max_pages_per_seq, storage, latent_quant)
         self._h = C.c_void_p()
         st = self.lib.kvcar_create(C.byref(self.cfg), C.byref(self._h))
         if st != 0:
@@ -295,6 +297,11 @@ class Context:
         off, pitch, width = C.c_size_t(), C.c_size_t(), C.c_int32()
         self._check(self.lib.kvcar_pool_layout(self._h, layer, which, C.byref(off), C.byref(pitch), C.byref(width)))
         return off.value, pitch.value, width.value
+
+    def pool_quant_layout(self, layer: int, which: int) -> int:
+        off = C.c_size_t()
+        self._check(self.lib.kvcar_pool_quant_layout(self._h, layer, which, C.byref(off)))
+        return off.value
 
     def cache_bytes_per_token(self) -> Tuple[float, float]:
         a, b = C.c_double(), C.c_double()

@@ -53,6 +53,8 @@ struct kvcar_ctx {
     char *pool = nullptr, *weights = nullptr, *ws = nullptr;
     std::vector<size_t> pool_off, cur_off;  // [layer*2+which]
     std::vector<int> width;                 // elements per row
+    std::vector<size_t> qparam_off;         // int8 latent rows: offset of the (scale, zero-point) array, else 0
+    std::vector<char> quant;                // [layer*2+which]: rows are int8 codes
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
     size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
     size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0, pfhid_off = 0;  // inside workspace
@@ -111,13 +113,22 @@ void compute_layout(kvcar_ctx *c) {
     c->pool_off.assign(nl * 2, 0);
     c->cur_off.assign(nl * 2, 0);
     c->width.assign(nl * 2, 0);
+    c->qparam_off.assign(nl * 2, 0);
+    c->quant.assign(nl * 2, 0);
     size_t off = 0;
     c->max_d = c->max_m = c->max_in = 0;
     for (int i = 0; i < nl * 2; ++i) {
         c->width[i] = stored_width(c, i / 2, i % 2);
         c->pool_off[i] = off;
-        off = align_up(off + rows * c->width[i] * c->elem, 256);
         const AEHost &a = c->ae[i];
+        if (g.latent_quant && a.set) {  // Eq. 4: one byte per element, then (scale, zero-point) per row
+            c->quant[i] = 1;
+            off = align_up(off + rows * c->width[i], 256);
+            c->qparam_off[i] = off;
+            off = align_up(off + rows * 2 * sizeof(float), 256);
+        } else {
+            off = align_up(off + rows * c->width[i] * c->elem, 256);
+        }
         if (a.set) {
             c->max_d = std::max(c->max_d, a.latent);
             c->max_m = std::max(c->max_m, a.hidden);
@@ -395,6 +406,17 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
     if (c->bound) return fail(c, KVCAR_ERR_STATE, "memory already bound");
     if (((uintptr_t)pool | (uintptr_t)weights | (uintptr_t)workspace) & 255)
         return fail(c, KVCAR_ERR_INVALID_ARG, "buffers must be 256-byte aligned");
+    if (c->cfg.latent_quant) {
+        if (c->cfg.storage != KVCAR_BF16) return fail(c, KVCAR_ERR_UNSUPPORTED, "int8 latent rows need bf16 storage");
+        for (int i = 0; i < c->cfg.n_layers * 2; ++i) {
+            const AEHost &a = c->ae[i];
+            if (!a.set && !stored_heads(c, i / 2, i % 2).empty())
+                return fail(c, KVCAR_ERR_UNSUPPORTED, "int8 latent rows need an autoencoder wherever heads are stored");
+            if (a.set && (a.latent % 16 != 0 || a.latent > a.in_dim))
+                return fail(c, KVCAR_ERR_UNSUPPORTED,
+                            "int8 latent rows need latent widths that are multiples of 16 and no wider than the input");
+        }
+    }
     compute_layout(c);
     if (pool_bytes < c->pool_bytes || weights_bytes < c->weights_bytes || workspace_bytes < c->ws_bytes)
         return fail(c, KVCAR_ERR_WORKSPACE, "a bound buffer is smaller than kvcar_required_bytes reports");
@@ -474,6 +496,7 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
                     sp.pool = c->pool + c->pool_off[idx];
                     sp.width = c->width[idx];
                     sp.compressed = a.set ? 1 : 0;
+                    sp.qparam = c->quant[idx] ? (const float *)(c->pool + c->qparam_off[idx]) : nullptr;
                     sp.n_need = 0;
                     if (a.set) {
                         sp.d = a.latent;
@@ -522,6 +545,7 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
         for (size_t k = 0; k < heads.size(); ++k) e.heads[k] = (int8_t)heads[k];
         e.in_dim = e.n_stored * hd;
         e.compressed = a.set ? 1 : 0;
+        e.qparam = c->quant[i] ? (float *)(c->pool + c->qparam_off[i]) : nullptr;
         if (a.set) {
             e.d = a.latent;
             e.m = a.hidden;
@@ -643,7 +667,7 @@ static kvcar_status enqueue_encode(kvcar_ctx *c, int32_t layer, const int32_t *s
     // one token per sequence: one launch per fully connected layer, features spread over all SMs
     // (needs 16-byte loadable weight rows and its row block in shared memory)
     const int vl = 16 / c->elem;
-    bool split_ok = n_tokens == 1 && c->cfg.head_dim % vl == 0 && encode_split_smem(c->max_in, c->max_m) <= 200 * 1024;
+    bool split_ok = n_tokens == 1 && !c->cfg.latent_quant && c->cfg.head_dim % vl == 0 && encode_split_smem(c->max_in, c->max_m) <= 200 * 1024;
     for (int w = 0; w < 2 && split_ok; ++w) {
         const AEHost &ae = c->ae[layer * 2 + w];
         if (ae.set && (ae.in_dim % vl || ae.hidden % vl)) split_ok = false;
@@ -666,8 +690,8 @@ kvcar_status kvcar_encode_append_tensor(kvcar_ctx *c, int32_t layer, const int32
     if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
     if (((uintptr_t)k | (uintptr_t)v) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "k/v must be 16-byte aligned");
     const kvcar_config &g = c->cfg;
-    if (g.storage != KVCAR_BF16 || g.head_dim != 64)
-        return fail(c, KVCAR_ERR_UNSUPPORTED, "the tensor-core encoder takes bf16 storage and 64-wide heads");
+    if (g.storage != KVCAR_BF16 || g.head_dim != 64 || g.latent_quant)
+        return fail(c, KVCAR_ERR_UNSUPPORTED, "the tensor-core encoder takes bf16 storage, bf16 latent rows and 64-wide heads");
     for (int w = 0; w < 2; ++w) {
         const AEHost &ae = c->ae[layer * 2 + w];
         if (!ae.set || ae.hidden % 16 || ae.latent % 16 || ae.hidden > 1024 || ae.latent > 1024)
@@ -916,14 +940,27 @@ kvcar_status kvcar_pool_layout(kvcar_ctx *c, int32_t layer, int32_t which, size_
     const int i = layer * 2 + which;
     *offset = c->pool_off[i];
     *width = c->width[i];
-    *row_pitch = (size_t)c->width[i] * c->elem;
+    *row_pitch = (size_t)c->width[i] * (c->quant[i] ? 1 : c->elem);
+    return KVCAR_OK;
+}
+
+kvcar_status kvcar_pool_quant_layout(kvcar_ctx *c, int32_t layer, int32_t which, size_t *param_offset) {
+    if (!c || !param_offset) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (layer < 0 || layer >= c->cfg.n_layers || (which & ~1)) return fail(c, KVCAR_ERR_INVALID_ARG, "index out of range");
+    if (!c->bound) compute_layout(c);
+    if (!c->quant[layer * 2 + which]) return fail(c, KVCAR_ERR_STATE, "this (layer, K/V) holds no int8 rows");
+    *param_offset = c->qparam_off[layer * 2 + which];
     return KVCAR_OK;
 }
 
 kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *c, double *compressed, double *uncompressed) {
     if (!c || !compressed || !uncompressed) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
     double comp = 0;
-    for (int i = 0; i < c->cfg.n_layers * 2; ++i) comp += (double)stored_width(c, i / 2, i % 2) * c->elem;
+    for (int i = 0; i < c->cfg.n_layers * 2; ++i) {
+        const int w = stored_width(c, i / 2, i % 2);
+        // int8 rows (Eq. 4): one byte per element plus the row's scale and zero-point, where anything is stored
+        comp += (c->cfg.latent_quant && c->ae[i].set) ? (w ? w + 8.0 : 0.0) : (double)w * c->elem;
+    }
     *compressed = comp;
     *uncompressed = 2.0 * c->cfg.n_layers * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
     return KVCAR_OK;
@@ -941,7 +978,10 @@ kvcar_status kvcar_layer_work_per_token(kvcar_ctx *c, int32_t layer, double *byt
             if (!need[s]) continue;
             const AEHost &a = c->ae[s * 2 + which];
             // a latent row mixes all heads of its layer and is read whole; of a raw row only the needed heads' slices
-            b += a.set ? (double)stored_width(c, s, which) * c->elem : (double)need[s] * hd * c->elem;
+            if (a.set && c->cfg.latent_quant)
+                b += stored_width(c, s, which) + 8.0;
+            else
+                b += a.set ? (double)stored_width(c, s, which) * c->elem : (double)need[s] * hd * c->elem;
             if (a.set) f += 2.0 * a.latent * a.hidden + 2.0 * a.hidden * hd * need[s];
         }
     }

@@ -135,9 +135,48 @@ __global__ void __launch_bounds__(256) encode_generic_kernel(const __grid_consta
             for (int r = 0; r < ER; ++r) acc[r] = fmaf(hs[r * m + k], w, acc[r]);
         }
         float b = pl.b2[j];
+        if (pl.qparam) {  // int8 rows: the whole row is needed before any code can be written
 #pragma unroll
-        for (int r = 0; r < ER; ++r)
-            if (rows[r] >= 0) st(pool + rows[r] * pl.width + j, acc[r] + b);
+            for (int r = 0; r < ER; ++r) xs[r * in_dim + j] = acc[r] + b;  // d <= in_dim (checked at bind time)
+        } else {
+#pragma unroll
+            for (int r = 0; r < ER; ++r)
+                if (rows[r] >= 0) st(pool + rows[r] * pl.width + j, acc[r] + b);
+        }
+    }
+    if (!pl.qparam) return;
+    // Eq. 4 per cached row: scale = 255/(max-min), zero-point = -round(scale*min) - 128,
+    // code = round(scale*x + zero-point) kept inside int8.  One warp per row (ER = warps per block).
+    __syncthreads();
+    const int r = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (rows[r] < 0) return;
+    const float *z = xs + r * in_dim;
+    float lo = INFINITY, hi = -INFINITY;
+    for (int j = lane; j < d; j += 32) {
+        lo = fminf(lo, z[j]);
+        hi = fmaxf(hi, z[j]);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    float scale, zp;
+    if (hi > lo) {
+        scale = 255.f / (hi - lo);
+        zp = -rintf(scale * lo) - 128.f;
+    } else {  // a row of equal values has no range: code 0 with zero-point -x restores it exactly
+        scale = 1.f;
+        zp = -lo;
+    }
+    int8_t *codes = reinterpret_cast<int8_t *>(pl.pool) + rows[r] * pl.width;
+    for (int j = lane; j < d; j += 32) {
+        float q = hi > lo ? fminf(fmaxf(rintf(fmaf(scale, z[j], zp)), -128.f), 127.f) : 0.f;
+        codes[j] = (int8_t)(int)q;
+    }
+    if (lane == 0) {
+        pl.qparam[rows[r] * 2] = scale;
+        pl.qparam[rows[r] * 2 + 1] = zp;
     }
 }
 
@@ -209,11 +248,24 @@ template <typename T>
 __device__ void hidden_tile(const SourcePlan &sp, const GenSmem &sm, const int64_t *rows, int valid) {
     const int tid = threadIdx.x;
     const T *pool = reinterpret_cast<const T *>(sp.pool);
-    for (int o = tid; o < sp.d * TOK; o += NT) {
-        int k = o % sp.d, t = o / sp.d;
-        float v = 0.f;
-        if (t < valid) v = ld(pool + rows[t] * sp.width + k);
-        sm.zT[k * TOK + t] = v;
+    if (sp.qparam) {  // int8 rows (Eq. 4, last line): x = (code - zero-point) / scale
+        const int8_t *codes = reinterpret_cast<const int8_t *>(sp.pool);
+        for (int o = tid; o < sp.d * TOK; o += NT) {
+            int k = o % sp.d, t = o / sp.d;
+            float v = 0.f;
+            if (t < valid) {
+                const float scale = sp.qparam[rows[t] * 2], zp = sp.qparam[rows[t] * 2 + 1];
+                v = ((float)codes[rows[t] * sp.width + k] - zp) / scale;
+            }
+            sm.zT[k * TOK + t] = v;
+        }
+    } else {
+        for (int o = tid; o < sp.d * TOK; o += NT) {
+            int k = o % sp.d, t = o / sp.d;
+            float v = 0.f;
+            if (t < valid) v = ld(pool + rows[t] * sp.width + k);
+            sm.zT[k * TOK + t] = v;
+        }
     }
     __syncthreads();
     const T *w1t = reinterpret_cast<const T *>(sp.w1t);

@@ -23,6 +23,7 @@ struct SourcePlan {
     const float *b2;   // [in_dim]
     const void *w1k;   // K-major bf16 copies for the tensor-core kernel: [m][d]
     const void *w2k;   //                                                  [in_dim][m]
+    const float *qparam;  // int8 rows: (scale, zero-point) per pool row, else null
     int32_t width;     // elements per pool row (= d if compressed, = in_dim if raw)
     int32_t d, m, in_dim;
     int32_t compressed;
@@ -55,6 +56,7 @@ struct EncPlan {
     const float *b2;
     const void *w1r;  // encoder FC1 as given, [m][in_dim], storage dtype (rows read by one warp each)
     const void *w2r;  // encoder FC2 as given, [d][m]
+    float *qparam;    // int8 rows: (scale, zero-point) per pool row, else null
     int32_t width, d, m, in_dim, compressed, n_stored;
     float slope;
     int32_t pad_;

@@ -1237,7 +1237,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
             const WhichPlan &wp = plans[l].w[which];
             for (int s = 0; s < wp.n_src && ok; ++s) {
                 const SourcePlan &sp = wp.src[s];
-                if (!sp.compressed || sp.d % 16 || sp.m % 16 || sp.d < 16 || sp.m < 16 || sp.m > 256 * MAX_HID_GROUPS || sp.in_dim > 256 * MAX_HID_GROUPS ||
+                if (!sp.compressed || sp.qparam /* int8 rows: generic kernel */ || sp.d % 16 || sp.m % 16 || sp.d < 16 || sp.m < 16 || sp.m > 256 * MAX_HID_GROUPS || sp.in_dim > 256 * MAX_HID_GROUPS ||
                     sp.in_dim % 64 || sp.width != sp.d) {
                     ok = false;
                     break;

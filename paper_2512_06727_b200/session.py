@@ -24,12 +24,13 @@ class Session:
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, page_tokens: int,
                  max_seqs: int, max_pages: int, max_pages_per_seq: int, storage: str,
                  src_k=None, src_v=None, autoencoders: Optional[Dict[Tuple[int, int], dict]] = None,
-                 device: str = "cuda:0", kernel: int = B.KERNEL_AUTO):
+                 device: str = "cuda:0", kernel: int = B.KERNEL_AUTO, latent_quant: bool = False):
         self.storage = storage_code(storage)
         self.dtype = torch_dtype(self.storage)
         self.device = torch.device(device)
         self.ctx = B.Context(n_layers, n_q_heads, n_kv_heads, head_dim, page_tokens, max_seqs, max_pages,
-                             max_pages_per_seq, self.storage)
+                             max_pages_per_seq, self.storage, int(latent_quant))
+        self.latent_quant = bool(latent_quant)
         if src_k is not None:
             self.ctx.set_reuse_map(src_k, src_v)
         for (layer, which), ae in (autoencoders or {}).items():
@@ -59,7 +60,15 @@ class Session:
         rows = self.ctx.cfg.max_pages * self.ctx.cfg.page_tokens
         base = self._aligned(self.pool) - self.pool.data_ptr() + off
         raw = self.pool[base:base + rows * pitch]
+        if pitch == width and self.latent_quant:   # int8 codes (Eq. 4)
+            return raw.view(torch.int8).view(rows, width)
         return raw.view(self.dtype).view(rows, width)
+
+    def pool_quant_params(self, layer: int, which: int) -> torch.Tensor:
+        """View of one layer's per-row (scale, zero-point) pairs [max_pages*page_tokens, 2] (int8 latent rows)."""
+        rows = self.ctx.cfg.max_pages * self.ctx.cfg.page_tokens
+        base = self._aligned(self.pool) - self.pool.data_ptr() + self.ctx.pool_quant_layout(layer, which)
+        return self.pool[base:base + rows * 8].view(torch.float32).view(rows, 2)
 
     def to_device(self, x: np.ndarray) -> torch.Tensor:
         return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(self.device).to(self.dtype).contiguous()

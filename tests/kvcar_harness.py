@@ -35,8 +35,11 @@ class Pair:
     def __init__(self, w: synth.Workload, max_seqs: int, max_pages: int, max_pages_per_seq: int,
                  src_k: Optional[np.ndarray] = None, src_v: Optional[np.ndarray] = None,
                  compressed_layers: Optional[List[int]] = None, compress: bool = True,
-                 kernel: int = B.KERNEL_AUTO, with_oracle: bool = True, ae_kwargs: Optional[dict] = None):
+                 kernel: int = B.KERNEL_AUTO, with_oracle: bool = True, ae_kwargs: Optional[dict] = None,
+                 latent_quant: bool = False):
+        """latent_quant: int8 latent rows (Eq. 4) on both sides; inputs and weights stay on w.storage's grid."""
         self.w = w
+        self.latent_quant = latent_quant
         n = w.n_layers * w.n_kv_heads
         if src_k is None:
             src_k = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
@@ -48,12 +51,13 @@ class Pair:
         self.o = None
         if with_oracle:
             self.o = KVCAROracle(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, max_seqs,
-                                 max_pages, w.storage)
+                                 max_pages, "int8" if latent_quant else w.storage)
             self.o.set_reuse_map(src_k, src_v)
             for (l, which), ae in self.aes.items():
                 self.o.set_autoencoder(l, which, ae)
         self.s = Session(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, max_seqs, max_pages,
-                         max_pages_per_seq, w.storage, src_k, src_v, self.aes, kernel=kernel)
+                         max_pages_per_seq, w.storage, src_k, src_v, self.aes, kernel=kernel,
+                         latent_quant=latent_quant)
         self.oracle_seqs: Optional[set] = None     # None = the oracle mirrors every sequence
 
     # ------------------------------------------------------------------
@@ -181,12 +185,39 @@ class Pair:
                     if self.o.stored_width(l, which) == 0:
                         continue
                     ref = self.o._pool(l, which)[rows]
+                    if self.latent_quant:
+                        worst = max(worst, self._check_int8_rows(l, which, rows, ref))
+                        continue
                     got = self.s.pool_rows(l, which)[torch.tensor(rows, device=self.s.device)].float().cpu().numpy()
                     err = np.abs(got - ref)
                     tol = latent_tol(w.storage, ref, bf16_hidden)
                     assert np.all(err <= tol), (l, which, s, float((err - tol).max()))
                     worst = max(worst, float(err.max()))
         return worst
+
+
+    def _check_int8_rows(self, l: int, which: int, rows, ref: np.ndarray) -> float:
+        """int8 rows: the oracle keeps each row as Eq. 4 returns it, x' = (q - zp)/scale with scale = 255/(max-min).
+        The library's latents carry fp32 rounding, so its row range, scale and zero-point differ by a few fp32 ulps
+        and a code may fall on the other side of a rounding boundary: a restored value may be off by one code step
+        (1/scale = range/255) plus the fp32 noise, never more.  The codes are int8 and the parameters finite."""
+        idx = torch.tensor(rows, device=self.s.device)
+        q = self.s.pool_rows(l, which)[idx]
+        assert q.dtype == torch.int8
+        par = self.s.pool_quant_params(l, which)[idx].cpu().numpy().astype(np.float64)
+        scale, zp = par[:, :1], par[:, 1:]
+        assert np.all(np.isfinite(par)) and np.all(scale > 0)
+        assert np.all(zp == np.rint(zp)), "zero-points are whole numbers (Eq. 4)"
+        got = (q.cpu().numpy().astype(np.float64) - zp) / scale
+        rng = ref.max(axis=1, keepdims=True) - ref.min(axis=1, keepdims=True)
+        # the oracle's row spans exactly 255 code steps
+        np.testing.assert_allclose(scale * rng, 255.0, rtol=1e-4)
+        err = np.abs(got - ref)
+        tol = 1.02 * rng / 255.0 + 1e-5
+        assert np.all(err <= tol), (l, which, float((err / tol).max()))
+        # and almost every code agrees: a step of difference only at a rounding boundary
+        assert np.mean(err > 0.02 * rng / 255.0 + 1e-5) < 0.02, (l, which, float(np.mean(err > 0.02 * rng / 255.0)))
+        return float(err.max())
 
 
 def assert_close(got: np.ndarray, ref: np.ndarray, storage: str, what=""):

@@ -353,3 +353,27 @@ def test_device_side_wait_that_runs_out_is_reported_and_the_context_stays_usable
     assert e.value.status == 7 and "0x7e57" in str(e.value)
     p.s.ctx.sync_status(p.s.stream())            # the word was cleared: reported once
     _check_step(p.decode_step([0, 1], 0), "bf16", "after a timed-out wait")
+
+
+@pytest.mark.parametrize("cfg", ["c2", "c3"])
+def test_int8_latent_rows_match_the_oracle(cfg):
+    """Sec. "Quantization" on top of the autoencoders (Table 5's combination): every cached latent row is stored
+    as int8 codes with its own scale and zero-point (Eq. 4) and restored before the decoder.  Cached rows are
+    compared as restored values (one code step at most, almost all equal), attention outputs at the bf16
+    tolerance, bytes per token exactly."""
+    w = synth.scaled(synth.CONFIGS[cfg], batch=3, cached_tokens=0, decode_steps=2)
+    p = Pair(w, max_seqs=4, max_pages=16, max_pages_per_seq=6, latent_quant=True)
+    seqs = [2, 0, 3]
+    p.open(seqs)
+    p.prefill([2], 200)
+    p.prefill([0], 131)
+    p.prefill([3], 1)
+    p.check_latents(seqs)
+    for step in range(2):
+        _check_step(p.decode_step(seqs, step), "bf16", f"int8 step {step}")
+    p.check_latents(seqs)
+    comp, full = p.s.ctx.cache_bytes_per_token()
+    assert (comp, full) == p.o.cache_bytes_per_token()
+    plain = Pair(w, max_seqs=1, max_pages=1, max_pages_per_seq=1, with_oracle=False)
+    assert comp < 0.55 * plain.s.ctx.cache_bytes_per_token()[0]
+

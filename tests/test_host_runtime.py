@@ -154,6 +154,37 @@ def test_accounting_and_layout():
     assert c1.layer_work_per_token(0) == (1536.0, 2654208.0 + 3072.0)
 
 
+def test_int8_latent_rows_accounting_and_layout():
+    """int8 latent rows (Sec. "Quantization", Eq. 4): one byte per element plus 8 bytes of scale and zero-point
+    per cached row and (layer, K/V); the library's bytes per token equal the oracle's, the codes' row pitch is the
+    width in bytes and the parameter array follows the codes, 256-byte aligned."""
+    for name in ("c2", "c3"):
+        w = synth.CONFIGS[name]
+        src = synth.make_reuse_map(w.n_layers, w.n_kv_heads, w.reuse_frac, w.seed)
+        o = KVCAROracle(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, 6, 40, "int8")
+        c = B.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, 6, 40, 12, B.BF16, 1)
+        o.set_reuse_map(src, src)
+        c.set_reuse_map(src, src)
+        for (l, which), ae in synth.make_stack_autoencoders(w, src, src).items():
+            o.set_autoencoder(l, which, ae)
+            c.set_autoencoder(l, which, ae)
+        assert c.cache_bytes_per_token() == o.cache_bytes_per_token()
+        rows = 40 * w.page_tokens
+        for l in range(w.n_layers):
+            for which in (K, V):
+                off, pitch, width = c.pool_layout(l, which)
+                assert width == o.stored_width(l, which) and pitch == width
+                if width:
+                    par = c.pool_quant_layout(l, which)
+                    assert par % 256 == 0 and par >= off + rows * pitch
+    # a stack with uncompressed stored rows cannot take int8 latent rows: bind refuses, nothing is launched
+    w = synth.CONFIGS["c2"]
+    c = B.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.page_tokens, 2, 4, 2, B.BF16, 1)
+    with pytest.raises(B.KvcarError) as e:
+        c.bind_memory(256, 1 << 20, 512, 1 << 20, 768, 1 << 20, 0)
+    assert e.value.status == 5
+
+
 def test_library_accounting_reproduces_the_printed_percentages():
     """The library's own kvcar_cache_bytes_per_token, driven through the C ABI, against the cache reductions the paper
     prints (Tables 2, 3 and 4; the records and their citations are in tests/golden/paper_accounting.txt)."""
