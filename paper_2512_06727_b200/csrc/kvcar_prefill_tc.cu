@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(PF_THREADS, 2)
     const uint32_t tmem = tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
+        if (elect_one()) {
             uint32_t phase = 0;
             for (int ks = 0; ks < n_slabs; ++ks) {
                 const int s = ks % PF_STAGES;
@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(PF_THREADS, 2)
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (elect_one()) {
             const uint32_t idesc = make_idesc(PF_M, nt);
             uint32_t phase = 0;
             for (int ks = 0; ks < n_slabs; ++ks) {

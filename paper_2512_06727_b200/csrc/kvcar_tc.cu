@@ -175,6 +175,35 @@ __device__ __forceinline__ void issue_kslab(uint32_t d_tmem, uint64_t a_desc, ui
     if (nk > 3) umma_pair<1>(d_tmem, a_desc + 6u, b_desc + 6u, idesc);
 }
 
+// ---------------------------------------------------------------------------- optional time stamps
+// Compile with -DKVCAR_TC_TRACE to make four threads of one cluster (lane 0 of the two producer warps, of the issuer
+// warp and of the first epilogue warp, in both CTAs) record (clock64 << 8) | tag at the points marked TR below;
+// kvcar_debug_trace_select picks the cluster, kvcar_debug_trace_dump fetches the records.  Without the macro the
+// marks compile to nothing.  Tags: producers 1 = pair begins, 2 = a hidden-chunk slab's two loads issued, 3 = a head
+// group slab's load issued; issuer 0x10 | kind = accumulator free, job begins, 0x30 = a slab's operands are in place,
+// 0x31 = its products and releases are issued, 0x19 = job committed; epilogue (kind << 4) | phase with kind 4 = hidden
+// chunk, 5 = K head group, 6 = V head group and phase 0 = waits for the job, 1 = job seen complete, 2 = accumulator
+// read and released, 3 = the job's epilogue is finished.
+#ifdef KVCAR_TC_TRACE
+constexpr int TRACE_LEN = 4096;
+__device__ unsigned long long g_trace[2][4][TRACE_LEN];
+__device__ int g_trace_n[2][4];
+__device__ int g_trace_cluster = 0;
+#define TR(role, tag)                                                                                          \
+    do {                                                                                                       \
+        if (tr_on) {                                                                                           \
+            if (tr_cnt < TRACE_LEN)                                                                            \
+                g_trace[rank][role][tr_cnt] = ((unsigned long long)clock64() << 8) | (unsigned)(tag);          \
+            ++tr_cnt;                                                                                          \
+            g_trace_n[rank][role] = tr_cnt < TRACE_LEN ? tr_cnt : TRACE_LEN;                                   \
+        }                                                                                                      \
+    } while (0)
+#else
+#define TR(role, tag) \
+    do {              \
+    } while (0)
+#endif
+
 // ---------------------------------------------------------------------------- the kernel
 // GMMA: query groups of more than two heads, whose attention products run on the warp-level tensor op (a separate
 // instantiation, so that the code of the other shapes carries none of it)
@@ -199,6 +228,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hq = a.hq, group = a.hq / a.hkv;
     const bool leader = rank == 0;
+#ifdef KVCAR_TC_TRACE
+    const bool tr_on = cid == g_trace_cluster && lane == 0 && (warp <= 2 || warp == PRODUCER2_WARP);
+    int tr_cnt = 0;
+#endif
 
     // carve shared memory (1024-byte aligned for the swizzled tiles; same offsets in both CTAs)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -266,10 +299,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // list are numbered and producer `pid` issues those of its parity.  Both walk the same sequence of
         // places and wait for each of them to be free, so both see the same ring state.
         const uint32_t pid = warp == 0 ? 0u : 1u;
-        if (lane == 0) {
+        if (elect_one()) {
             uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0;
           for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride) {
             const TileInfo mine = locate_tile(tix, 2 * pair + (int)rank, seqs.n);
+            TR(pid, 1);
             // pool rows of the tile's two 64-token halves (a half with no valid token re-reads a valid row block)
             int row[2] = {0, 0};
             if (mine.valid > 0) {
@@ -339,6 +373,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 tma_load_2d_pair(dst, sp.tm_w1, ks * 64, y0, fb);
                                 if (half_rows > 64) tma_load_2d_pair(dst + HALF_BYTES, sp.tm_w1, ks * 64, y0 + 64, fb);
                             }
+                            TR(pid, 2);
                         }
                     } else {
                         const int ks2 = (sp.m + 63) >> 6;
@@ -362,6 +397,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 if (yb >= 0)
                                     tma_load_2d_pair(s_ring + sl * SLOT_BYTES + HALF_BYTES, sp.tm_w2, ks * 64, yb, fb);
                             }
+                            TR(pid, 3);
                         }
                     }
                 }
@@ -370,9 +406,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         }
     } else if (warp == 1) {
         // ============================== MMA issuer (leader CTA) ==============================
-        // The whole warp walks the job list (warp-uniform control flow and operands); one lane issues.
-        if (leader) {
-            const bool issuer = lane == 0;
+        // One elected lane walks the job list and issues (the compiler then knows the branch holds a single thread
+        // and keeps descriptors and barrier addresses in uniform registers).
+        if (leader && elect_one()) {
+            constexpr bool issuer = true;
             uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0;
             const int ks_hid = (lay.max_m + 63) >> 6;
             auto wait_full = [&]() -> uint32_t {
@@ -393,6 +430,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     const uint32_t acc = tmem + 256u * buf;
                     mbar_wait(B.jempty + 8 * buf, ((jc >> 1) & 1u) ^ 1u, a.status, &abort_flag, 0x202);
                     tc_fence_after();
+                    TR(2, 0x10 | job.kind);
                     if (job.kind == 1) {
                         const int ks1 = (d + 63) >> 6;
                         const uint32_t idesc = make_idesc(256, job.nc);
@@ -418,11 +456,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             wait_full1(az, ez);
                             wait_full1(aw, ew2);
                             tc_fence_after();
+                            TR(2, 0x30);
                             if (issuer) {
                                 issue_kslab(acc, make_desc(az), make_desc(aw), idesc, min(4, (d - 64 * ks) >> 4), ks == 0);
                                 umma_commit_pair(ez);
                                 umma_commit_pair(ew2);
                             }
+                            TR(2, 0x31);
                         }
                     } else {
                         const int ks2 = (m + 63) >> 6;
@@ -442,6 +482,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             }
                             const uint32_t sw = wait_full();
                             tc_fence_after();
+                            TR(2, 0x30);
                             const uint64_t dh = make_desc(s_hidden + ks * SLOT_BYTES);
                             const uint64_t dw = make_desc(s_ring + sw * SLOT_BYTES);
                             const int nk = min(4, (m - 64 * ks) >> 4);
@@ -452,10 +493,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                     issue_kslab(acc, dw, dh, idesc, nk, ks == 0);
                                 umma_commit_pair(B.empty + 8 * sw);
                             }
+                            TR(2, 0x31);
                         }
                     }
                     if (issuer) umma_commit_pair(B.jfull + 8 * buf);
-                    __syncwarp();
+                    TR(2, 0x19);
                 }
             }
           }  // pairs
@@ -545,7 +587,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (GMMA) {
                     // this warp's probabilities are in place here; the peer's arrive as counted bytes, announced by one warp
                     __syncwarp();
-                    if (lane == 0) {
+                    if (elect_one()) {
                         if (ew == 0 && tl[rank ^ 1u].valid > 0)
                             mbar_expect_tx(B.p_ready, (uint32_t)nq_part * PBS * 2u);  // whole rows, see the softmax
                         else
@@ -555,7 +597,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     // every probability this CTA will read has been written, here and by the peer
                     asm volatile("fence.acq_rel.cluster;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0) {
+                    if (elect_one()) {
                         mbar_arrive_cluster(map_to_cta(B.p_ready, 0));
                         mbar_arrive_cluster(map_to_cta(B.p_ready, 1));
                     }
@@ -601,8 +643,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     // ---- bias + BatchNorm + LeakyReLU, bf16, into the swizzled hidden slabs ----
                     const float2 slope2 = make_float2(sp.slope, sp.slope);
                     const bool lr_max = sp.slope <= 1.f;
+                    TR(3, 0x40);
                     mbar_wait<false, 100>(B.jfull + 8 * buf, (jc >> 1) & 1u, a.status, &abort_flag, 0x301);
                     tc_fence_after();
+                    TR(3, 0x41);
                     // One 64-column slab at a time, this warp its half of it.  A hidden layer of a single chunk announces
                     // each slab as soon as it is written, so that the second layer's products start under the rest of
                     // this epilogue; a wider one announces each chunk once, through its last slab.
@@ -651,16 +695,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         if (slabwise) {
                             fence_async_smem();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive_remote(hid_leader + 8u * (uint32_t)((job.c0 >> 6) + sl));
+                            if (elect_one()) mbar_arrive_remote(hid_leader + 8u * (uint32_t)((job.c0 >> 6) + sl));
                         }
                     }
                     tc_fence_before();
                     if (!slabwise) fence_async_smem();
                     __syncwarp();
-                    if (lane == 0) {
+                    if (elect_one()) {
                         mbar_arrive_remote(jempty_leader[buf]);
                         if (!slabwise) mbar_arrive_remote(hid_leader + 8u * (uint32_t)((job.c0 >> 6) + nslabs - 1));
                     }
+                    TR(3, 0x43);
                     continue;
                 }
                 // ---- head group ----
@@ -728,8 +773,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         }
                     }
                 }
+                TR(3, 0x50 + 0x10 * which);
                 mbar_wait<false, 100>(B.jfull + 8 * buf, (jc >> 1) & 1u, a.status, &abort_flag, 0x302);
                 tc_fence_after();
+                TR(3, 0x51 + 0x10 * which);
                 if (SLAB && q_held) {  // every warp is past this pair's scores: the query rows are free
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
@@ -829,7 +876,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_remote(jempty_leader[buf]);
+                    if (elect_one()) mbar_arrive_remote(jempty_leader[buf]);
+                    TR(3, 0x52);
                     epi_bar_sync();
                     // tile softmax of the job's query heads; probabilities go to both CTAs.  A query group has several
                     // rows per warp: four per turn, so that their shuffle chains overlap
@@ -926,6 +974,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                          "r"(lay.epoch)
                                          : "memory");
                     }
+                    TR(3, 0x53);
                 } else {
                     // V: this thread owns (head place, channel) = row; columns = tokens of tile chalf
                     if (!lay.kv_split && !p_waited) {
@@ -1041,13 +1090,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_remote(jempty_leader[buf]);
+                    if (elect_one()) mbar_arrive_remote(jempty_leader[buf]);
+                    TR(3, 0x63);
                 }
             }
         }
         if (!lay.kv_split) {  // this CTA no longer reads the pair's probabilities: the peer may overwrite them
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(map_to_cta(B.s_free, rank ^ 1u));
+            if (elect_one()) mbar_arrive_remote(map_to_cta(B.s_free, rank ^ 1u));
         }
       }  // pairs
     }
@@ -1371,3 +1421,16 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
 }
 
 }  // namespace kvcar
+
+#ifdef KVCAR_TC_TRACE
+// Trace builds only: choose the cluster whose threads record, and fetch what they recorded
+// (out: [2 CTAs][4 roles][4096] entries of (clock64 << 8) | tag; n: entries per CTA and role).
+extern "C" int kvcar_debug_trace_select(int cluster) {
+    return (int)cudaMemcpyToSymbol(kvcar::g_trace_cluster, &cluster, sizeof(int));
+}
+extern "C" int kvcar_debug_trace_dump(unsigned long long *out, int *n) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, kvcar::g_trace, sizeof(kvcar::g_trace));
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(n, kvcar::g_trace_n, sizeof(kvcar::g_trace_n));
+    return (int)e;
+}
+#endif
