@@ -537,7 +537,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM bytes (read + write) per decode-kernel launch and listed sequence, from an ncu capture of the GPT-2-shaped
 # stack at 4096 cached tokens (batch 8, scaled by the batch: a launch's traffic is its sequences' latent rows)
-NCU_TRAFFIC = {"c5": {"bytes_per_sequence": 173.67e6 / 8, "captured_on": "c5_gpt2s_12l_L4096_b8",
+NCU_TRAFFIC = {"c5": {"bytes_per_sequence": 54.23e6 / 8, "captured_on": "c5_gpt2s_12l_L4096_b8",
                       "profile": "profiles/decode_pair_kernel_c5.md"}}
 
 

@@ -64,18 +64,19 @@ def lib_path() -> str:
 _LIB: Optional[C.CDLL] = None
 
 
-def load() -> C.CDLL:
-    """The library, built if its sources are newer, loaded once per process."""
+def load(trace: bool = False) -> C.CDLL:
+    """The library, built if its sources are newer, loaded once per process.  trace: the time-stamping build of
+    the same sources (must be the first load of the process)."""
     global _LIB
     if _LIB is None:
-        _LIB = _load()
+        _LIB = _load(trace)
     return _LIB
 
 
-def _load() -> C.CDLL:
-    path = lib_path()
-    if _build.needs_build():
-        _build.build()
+def _load(trace: bool = False) -> C.CDLL:
+    path = _build.TRACE_LIB if trace else lib_path()
+    if _build.needs_build(path):
+        _build.build(trace=trace)
     if not os.path.exists(path):
         raise ImportError(f"{path} is missing and could not be built; the CUDA library is required")
     lib = C.CDLL(path)
