@@ -45,6 +45,9 @@ def parse():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "tensor"])
     ap.add_argument("--uncompressed", action="store_true", help="raw K/V pages (the uncompressed twin)")
+    ap.add_argument("--absorbed", action="store_true",
+                    help="pass KVCAR_ABSORBED: K scores from the hidden vectors (absorbed last decoder layer); the roofline "
+                         "then counts that form's own, smaller number of operations")
     ap.add_argument("--api", default="fused", choices=["fused", "split"],
                     help="a layer's step through kvcar_step_layer (one call; the tile kernel runs beside the encoder) "
                          "or through kvcar_encode_append + kvcar_decode_attention")
@@ -597,7 +600,8 @@ def measure(w, args, torch, B, steps, warmup, uncompressed, flush, peaks, fused=
     fast_prefill(sess, w, torch)
     seqs = list(range(w.batch))
     stream = sess.stream()
-    flags = B.INCLUDE_CURRENT_EXACT
+    absorbed = bool(getattr(args, "absorbed", False)) and not uncompressed
+    flags = B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if absorbed else 0)
     n_in = 4
     k, v, q, out = step_inputs(sess, w, torch, n_in)       # a few input sets, cycled (values do not matter)
     for i in range(warmup):
@@ -633,10 +637,15 @@ def measure(w, args, torch, B, steps, warmup, uncompressed, flush, peaks, fused=
         sess.ctx.advance(seqs, 1, stream)
     torch.cuda.synchronize()
     sess.ctx.sync_status(stream)
-    flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
+    plain_flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
+    flops = sum(sess.ctx.layer_work_absorbed(l) * L * w.batch for (l, L, _, _) in kev) if absorbed else plain_flops
     byts = sum(sess.ctx.layer_work_per_token(l)[0] * L * w.batch for (l, L, _, _) in kev)
     kern_s = sum(a_.elapsed_time(b_) for (_, _, a_, b_) in kev) / 1e3
     roof = roofline_of(flops, byts, kern_s, peaks, len(kev))
+    if absorbed:   # the plain form's operations over the same time: what the absorbed form is worth as plain-form throughput
+        roof["form"] = "absorbed K scores (KVCAR_ABSORBED): achieved and frac count this form's own operations"
+        roof["plain_form_flops_per_launch"] = plain_flops / len(kev)
+        roof["plain_form_equivalent_frac"] = plain_flops / kern_s / 1e12 / roof["peak"] if roof.get("bound") == "tensor" else None
     comp, full = sess.ctx.cache_bytes_per_token()
     res = {"tokens_per_s": w.batch * steps / (total_ms / 1e3), "ms_per_step": total_ms / steps, "steps": steps,
            "roofline": roof, "cache_bytes_per_token": comp, "uncompressed_bytes_per_token": full, "launches": int(launches),
@@ -707,7 +716,7 @@ def main():
     sess, src, aes, k, v, q, out = head.pop("session")
     seqs = list(range(w.batch))
     stream = sess.stream()
-    flags = B.INCLUDE_CURRENT_EXACT
+    flags = B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if (args.absorbed and not args.uncompressed) else 0)
 
     # ---- e2e: host buffers through the C ABI, copies inside the timed region ----
     e2e = None
@@ -809,7 +818,8 @@ def main():
                            "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
                            "latent_full": 0 if args.uncompressed else w.latent_full, "reuse_frac": w.reuse_frac,
                            "page_tokens": w.page_tokens, "kernel": args.kernel, "api": args.api,
-                           "uncompressed": bool(args.uncompressed), "storage": w.storage,
+                           "uncompressed": bool(args.uncompressed), "absorbed": bool(args.absorbed and not args.uncompressed),
+                           "storage": w.storage,
                            "l2": "flushed between steps and between the per-launch timings (256 MiB write outside the event pairs)",
                            "cache_bytes_per_token": head["cache_bytes_per_token"],
                            "uncompressed_bytes_per_token": head["uncompressed_bytes_per_token"],

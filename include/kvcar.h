@@ -63,6 +63,7 @@ typedef enum {
 
 /* flags of kvcar_decode_attention */
 #define KVCAR_INCLUDE_CURRENT_EXACT 1u /* also attend to the current token through its exact K/V */
+#define KVCAR_ABSORBED 2u /* K side through the absorbed last decoder layer (see kvcar_decode_attention) */
 
 #define KVCAR_MAX_BATCH 512    /* sequences per launching call   */
 #define KVCAR_MAX_KV_HEADS 32
@@ -207,6 +208,14 @@ kvcar_status kvcar_advance(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, 
  * KVCAR_INCLUDE_CURRENT_EXACT the exact current-token K/V written by this
  * step's kvcar_encode_append of the root layer joins the attended set.
  * A sequence with nothing to attend to yields zeros.
+ * KVCAR_ABSORBED: the decoder ends in a plain fully connected layer (Sec.
+ * "Network Architecture": FC, BatchNorm, LeakyReLU, FC, nothing after it), so
+ * a head's score q.k' with k' = W4_h a + b4_h equals a.(W4_h^T q) + q.b4_h,
+ * where a is the token's activated hidden vector: the restored K rows are then
+ * never formed.  The same result up to rounding (W4_h^T q is rounded to the
+ * storage type once per sequence and head); honoured by the tensor-core kernel
+ * for K when the launch fills the machine, ignored (plain form computed) by
+ * every other kernel and for V.
  */
 kvcar_status kvcar_decode_attention(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                     const void *q, void *out, uint32_t flags, void *stream);
@@ -303,6 +312,11 @@ kvcar_status kvcar_cache_bytes_per_token(kvcar_ctx *ctx, double *compressed, dou
  * and passed through its first decoder layer once; of a raw row only the needed
  * heads' slices are read). */
 kvcar_status kvcar_layer_work_per_token(kvcar_ctx *ctx, int32_t layer, double *bytes, double *flops);
+/* The same count of floating-point operations for the KVCAR_ABSORBED form: on the K side the second decoder layer
+ * (2 m 64 per needed head) and the 2 * 64 of q.k' per query head are replaced by 2 m per query head (the score taken
+ * from the hidden vector); V side and bytes unchanged.  The per-sequence cost of W4_h^T q (m * 64 multiply-adds per
+ * query head and call, not per token) is left out. */
+kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *ctx, int32_t layer, double *flops);
 /* Number of kernels the library has launched so far on this context. */
 kvcar_status kvcar_launch_count(kvcar_ctx *ctx, int64_t *count);
 /* Kernel family (kvcar_kernel: GENERIC, TENSOR or RAW) that kvcar_decode_attention will use

@@ -18,6 +18,7 @@ F32, BF16 = 0, 1
 K, V = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TENSOR, KERNEL_RAW = 0, 1, 2, 3
 INCLUDE_CURRENT_EXACT = 1
+ABSORBED = 2
 MAX_BATCH = 512
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "STATE", 3: "OOM_PAGES", 4: "WORKSPACE", 5: "UNSUPPORTED",
@@ -29,7 +30,7 @@ EXPORTS = [
     "kvcar_encode_append", "kvcar_encode_append_tensor", "kvcar_advance", "kvcar_decode_attention", "kvcar_decode_attention_static",
     "kvcar_step_layer", "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout", "kvcar_pool_quant_layout",
-    "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
+    "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_layer_work_absorbed", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
     "kvcar_last_error", "kvcar_debug_expire_wait",
     "kvcar_head_l1_scratch_bytes", "kvcar_head_l1_distance", "kvcar_reuse_map_from_l1",
 ]
@@ -107,6 +108,7 @@ def _load(trace: bool = False) -> C.CDLL:
         "kvcar_pool_quant_layout": [vp, i32, i32, C.POINTER(sz)],
         "kvcar_cache_bytes_per_token": [vp, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "kvcar_layer_work_per_token": [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
+        "kvcar_layer_work_absorbed": [vp, i32, C.POINTER(C.c_double)],
         "kvcar_launch_count": [vp, C.POINTER(C.c_int64)],
         "kvcar_layer_kernel": [vp, i32, ip],
         "kvcar_sync_status": [vp, vp],
@@ -313,6 +315,11 @@ class Context:
         a, b = C.c_double(), C.c_double()
         self._check(self.lib.kvcar_layer_work_per_token(self._h, layer, C.byref(a), C.byref(b)))
         return a.value, b.value
+
+    def layer_work_absorbed(self, layer: int) -> float:
+        a = C.c_double()
+        self._check(self.lib.kvcar_layer_work_absorbed(self._h, layer, C.byref(a)))
+        return a.value
 
     def launch_count(self) -> int:
         n = C.c_int64()

@@ -57,7 +57,8 @@ struct kvcar_ctx {
     std::vector<char> quant;                // [layer*2+which]: rows are int8 codes
     size_t pool_bytes = 0, weights_bytes = 0, ws_bytes = 0;
     size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
-    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0, pfhid_off = 0;  // inside workspace
+    size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0, pfhid_off = 0, abs_off = 0;  // inside workspace
+    int max_k_sources = 0;  // most distinct source layers any layer's K heads resolve to
     std::vector<EncPlan> enc_host;  // the device's EncPlan table, host copy (tensor-core prefill builds tensor maps from it)
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
@@ -159,7 +160,7 @@ void compute_layout(kvcar_ctx *c) {
     c->enc_off = w;
     w = align_up(w + (size_t)nl * 2 * sizeof(EncPlan), 256);
     c->tmap_off = w;  // TMA descriptors of the tensor-core kernel: pool, decoder FC1, decoder FC2 per (layer, which)
-    w = align_up(w + (size_t)nl * 2 * 3 * 128, 256);
+    w = align_up(w + (size_t)nl * 2 * 3 * 128 + 128, 256);  // + the descriptor of the absorbed-score operands
     c->tcpart_off = w;  // per-layer job tables of the tensor-core kernel
     w = align_up(w + tc_part_bytes(nl), 256);
     c->weights_bytes = w;
@@ -186,6 +187,21 @@ void compute_layout(kvcar_ctx *c) {
     s = align_up(s + tc_split_bytes(g), 256);
     c->pfhid_off = s;  // bf16 hidden activations between the two launches of the tensor-core prefill
     if (g.storage == KVCAR_BF16 && c->max_m > 0) s = align_up(s + prefill_tc_scratch_bytes(c->max_m), 256);
+    c->max_k_sources = 0;
+    for (int l = 0; l < nl; ++l) {
+        std::vector<char> seen(nl, 0);
+        int n = 0;
+        for (int h = 0; h < g.n_kv_heads; ++h) {
+            const int r = resolve(c, l, h, 0).root_layer;
+            if (!seen[r]) {
+                seen[r] = 1;
+                ++n;
+            }
+        }
+        c->max_k_sources = std::max(c->max_k_sources, n);
+    }
+    c->abs_off = s;  // operands of the absorbed K scores (tensor-core kernel, KVCAR_ABSORBED)
+    s = align_up(s + tc_absorb_bytes(g, c->max_k_sources, c->max_m, nb), 256);
     c->ws_bytes = s;
 }
 
@@ -527,6 +543,11 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
     // tensor maps and job tables of the tensor-core kernel (fills their regions of the image)
     tc_setup(c->tc, c->cfg, plans, nl, c->weights, c->tmap_off, c->tcpart_off, img.data(),
              (size_t)g.max_pages * g.page_tokens);
+    {
+        const size_t slot = c->tmap_off + (size_t)nl * 2 * 3 * 128;
+        tc_setup_absorb(c->tc, c->cfg, c->max_k_sources, c->max_m, std::min(g.max_seqs, KVCAR_MAX_BATCH),
+                        c->ws + c->abs_off, img.data() + slot, c->weights + slot);
+    }
     c->tc.pbuf = reinterpret_cast<float *>(c->ws + c->kvsplit_off);
     c->tc.pflags = reinterpret_cast<uint32_t *>(c->ws + c->kvsplit_off +
                                                 (size_t)TC_SPLIT_TILES * g.n_q_heads * 132 * sizeof(float));
@@ -786,7 +807,9 @@ static kvcar_status enqueue_decode_tiles(kvcar_ctx *c, int32_t layer, const Deco
     } else if (want_tc) {
         int32_t lens[KVCAR_MAX_BATCH];
         for (int i = 0; i < sl.n; ++i) lens[i] = c->len[sl.id[i]];
-        e = tc_launch_decode(c->tc, a, sl, lens, layer, st);
+        int n_launches = 1;
+        e = tc_launch_decode(c->tc, a, sl, lens, layer, st, &n_launches);
+        if (e == cudaSuccess) c->launches += n_launches - 1;
     } else {
         if (decode_generic_smem(a.hq, a.hd, c->max_d, c->max_m) > 227 * 1024)
             return fail(c, KVCAR_ERR_UNSUPPORTED, "shape needs more shared memory than one SM has");
@@ -811,7 +834,7 @@ static kvcar_status check_decode_args(kvcar_ctx *c, int32_t layer, const int32_t
         return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
     if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
-    if (flags & ~KVCAR_INCLUDE_CURRENT_EXACT) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    if (flags & ~(KVCAR_INCLUDE_CURRENT_EXACT | KVCAR_ABSORBED)) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
     return KVCAR_OK;
 }
 
@@ -991,6 +1014,29 @@ kvcar_status kvcar_layer_work_per_token(kvcar_ctx *c, int32_t layer, double *byt
     return KVCAR_OK;
 }
 
+kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *c, int32_t layer, double *flops) {
+    if (!c || !flops || layer < 0 || layer >= c->cfg.n_layers) return fail(c, KVCAR_ERR_INVALID_ARG, "bad argument");
+    const int hkv = c->cfg.n_kv_heads, hd = c->cfg.head_dim, group = c->cfg.n_q_heads / hkv;
+    double f = 0;
+    for (int which = 0; which < 2; ++which) {
+        std::vector<int> need(c->cfg.n_layers, 0);
+        for (int h = 0; h < hkv; ++h) ++need[resolve(c, layer, h, which).root_layer];
+        for (int s = 0; s < c->cfg.n_layers; ++s) {
+            if (!need[s]) continue;
+            const AEHost &a = c->ae[s * 2 + which];
+            if (!a.set) {
+                if (which == 0) f += 2.0 * need[s] * group * hd;  // raw K rows: plain q.k
+                continue;
+            }
+            f += 2.0 * a.latent * a.hidden;
+            f += which == 0 ? 2.0 * a.hidden * need[s] * group : 2.0 * a.hidden * hd * need[s];
+        }
+    }
+    f += 2.0 * c->cfg.n_q_heads * hd;  // p.V
+    *flops = f;
+    return KVCAR_OK;
+}
+
 kvcar_status kvcar_launch_count(kvcar_ctx *c, int64_t *count) {
     if (!c || !count) return KVCAR_ERR_INVALID_ARG;
     *count = c->launches;
@@ -1079,7 +1125,7 @@ extern "C" kvcar_status kvcar_decode_attention_static(kvcar_ctx *c, int32_t laye
         return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
     if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
-    if (flags & ~KVCAR_INCLUDE_CURRENT_EXACT) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    if (flags & ~(KVCAR_INCLUDE_CURRENT_EXACT | KVCAR_ABSORBED)) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
     const kvcar_config &g = c->cfg;
     int max_len = 0;
     for (int i = 0; i < n_seqs; ++i) max_len = std::max(max_len, c->len[seqs[i]]);

@@ -159,6 +159,14 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
         : "memory");
 }
 
+// 32 lanes x 8 columns of fp32
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float *v) {
+    uint32_t *r = reinterpret_cast<uint32_t *>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
 // 32 lanes x 32 columns of fp32: thread i of the warp gets lane (base+i), columns col..col+31
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
     uint32_t *r = reinterpret_cast<uint32_t *>(v);
@@ -233,11 +241,11 @@ inline EncodeTiledFn tensor_map_encoder() {
 // bf16 matrix [rows][cols], `pitch` elements between rows -> descriptor with a [64 rows][64 cols] box, 128B swizzle,
 // zero fill outside
 inline bool encode_bf16_map(EncodeTiledFn fn, void *dst_host, const void *dev_ptr, uint64_t rows, uint64_t cols,
-                            uint64_t pitch) {
+                            uint64_t pitch, uint32_t box_rows = 64) {
     CUtensorMap m;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {pitch * 2};
-    cuuint32_t box[2] = {64, 64};
+    cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(dev_ptr), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -90,6 +90,10 @@ struct PairLaunch {
     uint32_t epoch;     // value a probability flag takes in this launch
     float *pbuf;        // [tile][hq][PSTRIDE] probabilities (+ sum at 128) in global memory
     uint32_t *pflags;   // [tile][hkv]
+    // absorbed K scores (job kind 3): rows of W4_h^T q per (K source, listed sequence, query head), q.b4_h beside them
+    const void *tm_wq;  // TMA descriptor: box = 64 columns x nq_pad rows
+    const float *qbias; // [source][abs_batch][nq_pad]
+    int32_t nq_pad, abs_batch;
 };
 
 // ---------------------------------------------------------------------------- waits
@@ -375,6 +379,25 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             }
                             TR(pid, 2);
                         }
+                    } else if (job.kind == 3) {
+                        // absorbed scores: the column operand is this tile's sequence's W4_h^T q rows (all query heads)
+                        const int ks2 = (sp.m + 63) >> 6;
+                        const int y = ((int)job.src * lay.abs_batch + mine.si) * lay.nq_pad;
+                        const uint32_t slab_bytes = (uint32_t)lay.nq_pad * 128u;  // one K slab of this CTA's rows
+                        const int per_place = SLOT_BYTES / (int)slab_bytes;        // K slabs staged behind one barrier
+                        for (int ks0 = 0; ks0 < ks2; ks0 += per_place) {
+                            const int n = min(per_place, ks2 - ks0);
+                            const bool own = turn == pid;
+                            turn ^= 1u;
+                            const uint32_t sl = acquire(2u * slab_bytes * (uint32_t)n, own);
+                            if (own) {
+                                const uint32_t fb = map_to_cta(B.full + 8 * sl, 0);
+                                for (int i = 0; i < n; ++i)
+                                    tma_load_2d_pair(s_ring + sl * SLOT_BYTES + (uint32_t)i * slab_bytes, lay.tm_wq,
+                                                     (ks0 + i) * 64, y, fb);
+                            }
+                            TR(pid, 3);
+                        }
                     } else {
                         const int ks2 = (sp.m + 63) >> 6;
                         int ya, yb = -1;  // first rows of the one or two 64-row boxes this CTA supplies
@@ -462,6 +485,34 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 umma_commit_pair(ez);
                                 umma_commit_pair(ew2);
                             }
+                            TR(2, 0x31);
+                        }
+                    } else if (job.kind == 3) {
+                        // absorbed scores: the whole job's column operand is a few KB, so several K slabs share a place
+                        // and a barrier round; the waits for the activations are those of a first head group
+                        const int ks2 = (m + 63) >> 6;
+                        const uint32_t idesc = make_idesc(256, 2 * lay.nq_pad);
+                        const uint32_t slab_bytes = (uint32_t)lay.nq_pad * 128u;
+                        const int per_place = SLOT_BYTES / (int)slab_bytes;
+                        constexpr bool slabwise = SLAB;
+                        for (int ks0 = 0; ks0 < ks2; ks0 += per_place) {
+                            const int n = min(per_place, ks2 - ks0);
+                            for (int ks = ks0; ks < ks0 + n; ++ks)
+                                if (slabwise || (ks & 3) == 0) {
+                                    const int ws = slabwise ? ks : min(ks + 3, ks2 - 1);
+                                    mbar_wait(B.hid_ready + 8 * ws, (hid_phase >> ws) & 1u, a.status, &abort_flag, 0x204);
+                                    hid_phase ^= 1u << ws;
+                                }
+                            const uint32_t sw = wait_full();
+                            tc_fence_after();
+                            TR(2, 0x30);
+                            for (int i = 0; i < n; ++i) {
+                                const int ks = ks0 + i;
+                                issue_kslab(acc, make_desc(s_hidden + ks * SLOT_BYTES),
+                                            make_desc(s_ring + sw * SLOT_BYTES + (uint32_t)i * slab_bytes), idesc,
+                                            min(4, (m - 64 * ks) >> 4), ks == 0);
+                            }
+                            umma_commit_pair(B.empty + 8 * sw);
                             TR(2, 0x31);
                         }
                     } else {
@@ -787,7 +838,25 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (which == 0) {
                     // K: this thread owns token `row` of this CTA's tile; columns = (head place, channel)
                     const int nh = job.nh;
-                    if (GMMA) {
+                    if (job.kind == 3) {
+                        // absorbed scores: the accumulator already holds a.(W4_h^T q) for every query head of both
+                        // tiles' sequences; this CTA's sequence owns columns [nq_pad * rank, nq_pad * (rank + 1))
+                        const int half = lay.nq_pad >> 1;
+                        const uint32_t mask = (uint32_t)job.c0 | ((uint32_t)job.nc << 16);
+                        const float *qb_ = lay.qbias + ((size_t)job.src * lay.abs_batch + mine.si) * lay.nq_pad;
+                        for (int c8 = 0; c8 < half; c8 += 8) {
+                            const int c_lo = chalf * half + c8;
+                            float sc[8];
+                            tmem_ld8(acc + (uint32_t)(lay.nq_pad * (int)rank + c_lo), sc);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                const int ql = c_lo + c;
+                                if ((mask >> ql) & 1u)
+                                    Smine[ql * PSTRIDE + row] = row < mine.valid ? sc[c] + __ldg(qb_ + ql) : -INFINITY;
+                            }
+                        }
+                    } else if (GMMA) {
                         // scores of a query group as a small matrix product on the warp-level tensor op: the restored
                         // K rows come out of tensor memory already in the A-fragment layout (16 tokens x 16 channels per
                         // step), the group's queries are the B operand, one 16-token half of the warp's rows at a time
@@ -883,7 +952,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     // rows per warp: four per turn, so that their shuffle chains overlap
                     if (mine.valid > 0) {
                         constexpr int R = GMMA ? 4 : 1;
-                        const int n_items = nh * group;
+                        const int n_items = job.kind == 3 ? (int)P.abs_n[job.src] : nh * group;
                         for (int base = ew; base < n_items; base += R * N_EPI_WARPS) {
                             int qlv[R];
                             float4 sc[R];
@@ -895,7 +964,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 sc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 if (item < n_items) {
                                     const int hp = (int)(((uint32_t)item * ginv) >> 16);  // item / group
-                                    qlv[u] = (job_kvh(job, hp) - h_lo) * group + (item - hp * group);
+                                    qlv[u] = job.kind == 3 ? (int)P.abs_q[job.src][item]
+                                                           : (job_kvh(job, hp) - h_lo) * group + (item - hp * group);
                                     sc[u] = *reinterpret_cast<const float4 *>(Smine + qlv[u] * PSTRIDE + 4 * lane);
                                 }
                                 mx[u] = fmaxf(fmaxf(sc[u].x, sc[u].y), fmaxf(sc[u].z, sc[u].w));
@@ -1152,7 +1222,9 @@ int pick_nslot(int nq_local, int group, int max_m, int max_in, int pslots) {
 }
 
 // Job tables of one head subset [h_lo, h_hi) of one layer.  Returns false if it does not fit the table limits.
-bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int h_hi, TcPart &out) {
+// absorbed: the K head groups of every source are replaced by one score job over all its query heads (kind 3).
+bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int h_hi, TcPart &out, bool absorbed = false,
+                int group = 1) {
     memset(&out, 0, sizeof(out));
     out.h_lo = h_lo;
     out.h_hi = h_hi;
@@ -1184,6 +1256,23 @@ bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int
                 first = false;
             }
             first = true;
+            if (absorbed && which == 0) {
+                if (nj == TC_MAX_JOBS || (h_hi - h_lo) * group > TC_ABS_MAX_Q) return false;
+                TcJob &jb = out.jobs[which][nj++];
+                jb.kind = 3;
+                jb.src = (uint8_t)ns;
+                jb.first = 1;
+                uint32_t mask = 0;
+                for (int i = 0; i < n; ++i)
+                    for (int g = 0; g < group; ++g) mask |= 1u << ((heads[i] - h_lo) * group + g);
+                jb.c0 = (uint16_t)(mask & 0xffffu);
+                jb.nc = (uint16_t)(mask >> 16);
+                int cnt = 0;
+                for (int ql = 0; ql < TC_ABS_MAX_Q; ++ql)
+                    if ((mask >> ql) & 1u) out.abs_q[ns][cnt++] = (uint8_t)ql;
+                out.abs_n[ns] = (uint8_t)cnt;
+                n = 0;  // no head groups
+            }
             for (int i = 0; i < n;) {  // head groups: K 4/2/1 real heads; V always four places, padded
                 if (nj == TC_MAX_JOBS) return false;
                 TcJob &jb = out.jobs[which][nj++];
@@ -1245,7 +1334,72 @@ cudaError_t tc_launch_expire_wait(int32_t *status, uint64_t limit_ns, cudaStream
     return cudaGetLastError();
 }
 
-size_t tc_part_bytes(int n_layers) { return (size_t)n_layers * 7 * sizeof(TcPart); }
+// ---------------------------------------------------------------------------- absorbed K scores: operands
+// scores of head h against a token = a . (W4_h^T q) + q . b4_h with a the token's activated hidden vector (the
+// decoder's last layer is linear).  One block per (query head, listed sequence) forms the m-vector W4_h^T (q * scale)
+// as a bf16 row - the column operand of the score job - and the scalar q . b4_h.  W4 is the K-major copy
+// [in_dim][m], so consecutive threads read consecutive hidden columns.
+__global__ void __launch_bounds__(128) absorb_q_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ SeqList seqs,
+                                                       __nv_bfloat16 *wq, float *qbias, int nq_pad, int m_pad, int batch) {
+    __shared__ float qsm[64];
+    const int qh = blockIdx.x, si = blockIdx.y, tid = threadIdx.x;
+    const int kvh = qh / (a.hq / a.hkv);
+    const WhichPlan &wp = a.plan->w[0];
+    int s = 0, slot = 0;
+    for (int i = 0; i < wp.n_src; ++i)
+        for (int k = 0; k < wp.src[i].n_need; ++k)
+            if (wp.src[i].kv_head[k] == kvh) {
+                s = i;
+                slot = wp.src[i].slot[k];
+            }
+    const SourcePlan &sp = wp.src[s];
+    if (tid < 64)
+        qsm[tid] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.q)[((int64_t)si * a.hq + qh) * 64 + tid]) * a.scale;
+    __syncthreads();
+    const __nv_bfloat16 *w2 = reinterpret_cast<const __nv_bfloat16 *>(sp.w2k) + (int64_t)slot * 64 * sp.m;
+    __nv_bfloat16 *row = wq + (((int64_t)s * batch + si) * nq_pad + qh) * m_pad;
+    for (int j = tid; j < m_pad; j += 128) {
+        float acc = 0.f;
+        if (j < sp.m) {
+#pragma unroll 8
+            for (int c = 0; c < 64; ++c) acc = fmaf(__bfloat162float(w2[(int64_t)c * sp.m + j]), qsm[c], acc);
+        }
+        row[j] = __float2bfloat16_rn(acc);
+    }
+    if (tid < 32) {
+        float b = qsm[tid] * sp.b2[slot * 64 + tid] + qsm[tid + 32] * sp.b2[slot * 64 + tid + 32];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xffffffffu, b, o);
+        if (tid == 0) qbias[((int64_t)s * batch + si) * nq_pad + qh] = b;
+    }
+}
+
+size_t tc_absorb_bytes(const kvcar_config &cfg, int max_k_sources, int max_m, int batch) {
+    if (cfg.storage != KVCAR_BF16 || cfg.n_q_heads > TC_ABS_MAX_Q || max_k_sources <= 0 || max_m <= 0) return 0;
+    const size_t nq_pad = cfg.n_q_heads <= 16 ? 16 : 32, m_pad = ((size_t)max_m + 63) / 64 * 64;
+    const size_t rows = (size_t)max_k_sources * batch * nq_pad;
+    return (rows * m_pad * 2 + 255) / 256 * 256 + rows * sizeof(float);
+}
+
+void tc_setup_absorb(TcState &tc, const kvcar_config &cfg, int max_k_sources, int max_m, int batch, char *ws_area,
+                     char *tmap_host, char *tmap_dev) {
+    tc.wq = nullptr;
+    if (!tc.available || tc_absorb_bytes(cfg, max_k_sources, max_m, batch) == 0) return;
+    EncodeTiledFn fn = tensor_map_encoder();
+    if (!fn) return;
+    const int nq_pad = cfg.n_q_heads <= 16 ? 16 : 32, m_pad = (max_m + 63) / 64 * 64;
+    const size_t rows = (size_t)max_k_sources * batch * nq_pad;
+    if (!encode_bf16_map(fn, tmap_host, ws_area, rows, (uint64_t)m_pad, (uint64_t)m_pad, (uint32_t)nq_pad)) return;
+    tc.wq = ws_area;
+    tc.qbias = reinterpret_cast<float *>(ws_area + (rows * m_pad * 2 + 255) / 256 * 256);
+    tc.tm_wq = tmap_dev;
+    tc.abs_nq_pad = nq_pad;
+    tc.abs_m_pad = m_pad;
+    tc.abs_batch = batch;
+    tc.abs_max_src = max_k_sources;
+}
+
+size_t tc_part_bytes(int n_layers) { return (size_t)n_layers * TC_PARTS_PER_LAYER * sizeof(TcPart); }
 size_t tc_split_bytes(const kvcar_config &cfg) {
     return (size_t)TC_SPLIT_TILES * ((size_t)cfg.n_q_heads * PSTRIDE * sizeof(float) + (size_t)cfg.n_kv_heads * sizeof(uint32_t));
 }
@@ -1320,7 +1474,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
             }
         }
         if (!ok || max_m == 0) continue;
-        TcPart *parts = reinterpret_cast<TcPart *>(img + part_off) + (size_t)l * 7;
+        TcPart *parts = reinterpret_cast<TcPart *>(img + part_off) + (size_t)l * TC_PARTS_PER_LAYER;
         TcLayerCfg &lc = tc.layer[l];
         // hidden layers of a single chunk: every source keeps its parameter block in shared memory (see SLAB)
         const int pslots = max_m <= 256 ? plans[l].w[0].n_src + plans[l].w[1].n_src : 1;
@@ -1335,6 +1489,8 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
             lc.split_ok[si] = fits ? 1 : 0;
         }
         if (!lc.split_ok[0]) continue;
+        lc.abs_ok = cfg.n_q_heads <= TC_ABS_MAX_Q &&
+                    build_part(plans[l], srcs, 0, cfg.n_kv_heads, parts[TC_PARTS_PER_LAYER - 1], true, group) ? 1 : 0;
         lc.ok = 1;
         lc.max_m = (uint16_t)max_m;
         lc.max_in = (uint16_t)max_in;
@@ -1356,7 +1512,8 @@ bool tc_layer_supported(const TcState &tc, int layer) {
 }
 
 cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &seqs, const int32_t *lens,
-                             int layer, cudaStream_t st) {
+                             int layer, cudaStream_t st, int *n_launches) {
+    *n_launches = 1;
     const TcLayerCfg &lc = tc.layer[layer];
     TileIndex tix;
     uint32_t t = 0;
@@ -1396,7 +1553,20 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     lay.epoch = ++tc.epoch;
     lay.pbuf = tc.pbuf;
     lay.pflags = tc.pflags;
-    lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * 7 + part_index(split, 0);
+    lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * TC_PARTS_PER_LAYER + part_index(split, 0);
+    // the absorbed K form: only where one cluster takes a pair's whole layer (no head or K/V split)
+    if ((a.flags & KVCAR_ABSORBED) && lc.abs_ok && tc.wq && split == 1 && !kv_split && seqs.n <= tc.abs_batch) {
+        absorb_q_kernel<<<dim3(a.hq, seqs.n), 128, 0, st>>>(a, seqs, reinterpret_cast<__nv_bfloat16 *>(tc.wq), tc.qbias,
+                                                            tc.abs_nq_pad, tc.abs_m_pad, tc.abs_batch);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        *n_launches = 2;
+        lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * TC_PARTS_PER_LAYER + TC_PARTS_PER_LAYER - 1;
+        lay.tm_wq = tc.tm_wq;
+        lay.qbias = tc.qbias;
+        lay.nq_pad = tc.abs_nq_pad;
+        lay.abs_batch = tc.abs_batch;
+    }
     // never less than half an SM's shared memory: two CTAs on one SM would both want all of tensor memory
     const int smem = (int)std::max(launch_bytes(lay), 120u * 1024u);
     // at most one resident cluster per SM pair; clusters walk the pairs with that stride

@@ -110,11 +110,12 @@ class Pair:
             self.append(l, seqs, k, v, tensor=tensor)
         self.advance(seqs, n_tokens)
 
-    def attention(self, layer: int, seqs: Sequence[int], q: np.ndarray, include_current: bool = True):
+    def attention(self, layer: int, seqs: Sequence[int], q: np.ndarray, include_current: bool = True,
+                  absorbed: bool = False):
         """Returns (gpu [n,Hq,hd] float64, oracle rows or None, row indices the oracle covers)."""
         dq = self.s.to_device(q)
         out = torch.empty_like(dq)
-        flags = B.INCLUDE_CURRENT_EXACT if include_current else 0
+        flags = (B.INCLUDE_CURRENT_EXACT if include_current else 0) | (B.ABSORBED if absorbed else 0)
         self.s.ctx.decode_attention(layer, list(seqs), dq.data_ptr(), out.data_ptr(), flags, self.s.stream())
         self.s.ctx.sync_status(self.s.stream())
         got = out.float().cpu().numpy().astype(np.float64)
@@ -126,11 +127,11 @@ class Pair:
         return got, ref, rows
 
     def step_layer(self, layer: int, seqs: Sequence[int], k: np.ndarray, v: np.ndarray, q: np.ndarray,
-                   include_current: bool = True):
+                   include_current: bool = True, absorbed: bool = False):
         """append + attention of one layer through the single-call entry point; same return as attention()."""
         dk, dv, dq = self.s.to_device(k), self.s.to_device(v), self.s.to_device(q)
         out = torch.empty_like(dq)
-        flags = B.INCLUDE_CURRENT_EXACT if include_current else 0
+        flags = (B.INCLUDE_CURRENT_EXACT if include_current else 0) | (B.ABSORBED if absorbed else 0)
         self.s.ctx.step_layer(layer, list(seqs), dk.data_ptr(), dv.data_ptr(), dq.data_ptr(), out.data_ptr(), flags,
                               self.s.stream())
         self.s.ctx.sync_status(self.s.stream())
@@ -145,7 +146,7 @@ class Pair:
         return got, ref, rows
 
     def decode_step(self, seqs: Sequence[int], step: int, q_scale: float = 1.0, include_current: bool = True,
-                    layers: Optional[Sequence[int]] = None, fused: bool = False):
+                    layers: Optional[Sequence[int]] = None, fused: bool = False, absorbed: bool = False):
         """One full decode step (encode-append + attention for every layer, then
         advance).  Returns per-layer (gpu, oracle, rows).  fused: each layer through
         the single-call entry point instead of the two calls."""
@@ -157,12 +158,12 @@ class Pair:
             v = np.stack([synth.make_kv(w, l, V, s, t[s], 1) for s in seqs])
             if fused:
                 q = np.stack([synth.make_q(w, l, s, step, scale=q_scale) for s in seqs])
-                res[l] = self.step_layer(l, seqs, k, v, q, include_current)
+                res[l] = self.step_layer(l, seqs, k, v, q, include_current, absorbed)
                 continue
             self.append(l, seqs, k, v)
             if layers is None or l in layers:
                 q = np.stack([synth.make_q(w, l, s, step, scale=q_scale) for s in seqs])
-                res[l] = self.attention(l, seqs, q, include_current)
+                res[l] = self.attention(l, seqs, q, include_current, absorbed)
         self.advance(seqs, 1)
         return res
 

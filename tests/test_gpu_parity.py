@@ -377,3 +377,38 @@ def test_int8_latent_rows_match_the_oracle(cfg):
     plain = Pair(w, max_seqs=1, max_pages=1, max_pages_per_seq=1, with_oracle=False)
     assert comp < 0.55 * plain.s.ctx.cache_bytes_per_token()[0]
 
+
+@pytest.mark.parametrize("shape", ["gpt2", "tinyllama", "group2_narrow"])
+def test_absorbed_last_layer_matches_the_oracle(shape):
+    """KVCAR_ABSORBED: a head's scores are taken as a.(W4_h^T q) + q.b4_h from the activated hidden vectors, the
+    restored K rows are never formed (the decoder ends in a bare fully connected layer, Sec. "Network Architecture").
+    Same result as the plain form up to rounding: compared with the oracle at the usual tolerance on grids large
+    enough for the form to be taken, with reuse (several source layers per layer), and the launch counter shows that
+    the operand kernel ran."""
+    if shape == "gpt2":            # 12 heads, hidden 576 (three chunks), CUDA-core attention products
+        w = synth.scaled(synth.CONFIGS["c2"], n_layers=3, batch=5, cached_tokens=0, decode_steps=2, reuse_frac=0.25)
+    elif shape == "tinyllama":     # 32 query / 4 KV heads, hidden 192, tensor-op attention products
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, batch=5, cached_tokens=0, decode_steps=2, reuse_frac=0.25)
+    else:                          # 8 query / 4 KV heads
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, n_q_heads=8, n_kv_heads=4, latent_full=128, batch=5,
+                         cached_tokens=0, decode_steps=2, reuse_frac=0.25)
+    pps = 34
+    p = Pair(w, max_seqs=5, max_pages=5 * pps, max_pages_per_seq=pps, kernel=B.KERNEL_TENSOR)
+    seqs = [0, 1, 2, 3, 4]
+    p.open(seqs)
+    for s_, n in zip(seqs, (2100, 2049, 2111, 2050, 2064)):     # 17 tiles each: 85 tiles, 43 pairs
+        p.prefill([s_], n)
+    for step in range(2):
+        before = p.s.ctx.launch_count()
+        res = p.decode_step(seqs, step, absorbed=True)
+        # per layer: two encoder launches, the operand kernel, the tile kernel, the combine kernel (+ table updates)
+        assert p.s.ctx.launch_count() - before >= 5 * w.n_layers
+        _check_step(res, "bf16", f"absorbed {shape} step {step}")
+    # the flag is a no-op where the form is not taken (a grid small enough for the K/V split): same tolerance
+    w2 = synth.scaled(w, batch=2)
+    p2 = Pair(w2, max_seqs=2, max_pages=8, max_pages_per_seq=4, kernel=B.KERNEL_TENSOR)
+    p2.open([0, 1])
+    p2.prefill([0], 200)
+    p2.prefill([1], 130)
+    _check_step(p2.decode_step([0, 1], 0, absorbed=True), "bf16", f"absorbed flag on a small grid, {shape}")
+

@@ -364,6 +364,32 @@ def test_linear_decoder_identity():
         assert np.max(np.abs(e / e.sum() - probs[qh])) < 1e-12
 
 
+def test_absorbed_last_layer_identity_with_the_nonlinear_decoder():
+    """The decoder ends in a bare fully connected layer (Sec. "Network Architecture"), so with the usual LeakyReLU
+    slope the score q.k' of a restored key k' = W4_h a + b4_h equals a.(W4_h^T q) + q.b4_h, a being the token's
+    activated hidden vector.  The hidden vector is rebuilt here from the cached latents with plain numpy (not the
+    oracle's decoder) and the softmax over the absorbed scores must reproduce the oracle's probabilities."""
+    o = small_stack(2, 4, 2, 8, 4, 2, 8, "exact", reuse=[(K, 1, 0, 0), (V, 1, 1, 1)], seed=29)
+    fed, g = fill(o, [0], 7)
+    q = g.standard_normal((1, 4, 8))
+    for layer in range(2):
+        out, probs = o.decode_attention(layer, [0], q, include_current=False, return_probs=True)
+        rows = [o.locate(0, t)[1] for t in range(7)]
+        for qh in range(4):
+            kvh = qh // 2
+            root, head, slot = o.resolve(layer, kvh, K)
+            ae = o.ae[(root, K)]
+            gam, bet, mu, var = (np.asarray(r, np.float64) for r in ae["dec_bn"])
+            pre = o.pool[(root, K)][rows] @ np.asarray(ae["dec_w1"], np.float64).T + np.asarray(ae["dec_b1"], np.float64)
+            pre = (pre - mu) / np.sqrt(var + ae["bn_eps"]) * gam + bet
+            act = np.where(pre >= 0, pre, ae["leaky_slope"] * pre)                       # [tokens][m]
+            w4 = np.asarray(ae["dec_w2"], np.float64)[slot * 8:(slot + 1) * 8]
+            b4 = np.asarray(ae["dec_b2"], np.float64)[slot * 8:(slot + 1) * 8]
+            s_ = (act @ (w4.T @ q[0, qh]) + b4 @ q[0, qh]) / math.sqrt(8)
+            e = np.exp(s_ - s_.max())
+            assert np.max(np.abs(e / e.sum() - probs[qh])) < 1e-12, (layer, qh)
+
+
 # ---------------------------------------------------------------- pages
 def test_page_allocation_order_and_locate():
     o = KVCAROracle(1, 1, 1, 8, 4, 4, 6, "exact")
