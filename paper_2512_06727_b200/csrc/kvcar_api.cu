@@ -59,6 +59,7 @@ struct kvcar_ctx {
     size_t plan_off = 0, enc_off = 0, tmap_off = 0, tcpart_off = 0;  // inside weights
     size_t bt_off = 0, len_off = 0, status_off = 0, part_off = 0, stage_off = 0, enchid_off = 0, kvsplit_off = 0, pfhid_off = 0, abs_off = 0;  // inside workspace
     int max_k_sources = 0;  // most distinct source layers any layer's K heads resolve to
+    bool raw_maps = false;  // every raw bf16 pool has its TMA descriptor (raw-row kernel stages with tensor loads)
     std::vector<EncPlan> enc_host;  // the device's EncPlan table, host copy (tensor-core prefill builds tensor maps from it)
     int max_chunks = 0, chunk_tokens = 128;
     int max_d = 0, max_m = 0, max_in = 0;
@@ -548,6 +549,13 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
         tc_setup_absorb(c->tc, c->cfg, c->max_k_sources, c->max_m, std::min(g.max_seqs, KVCAR_MAX_BATCH),
                         c->ws + c->abs_off, img.data() + slot, c->weights + slot);
     }
+    // descriptors of the raw pools (their three slots are otherwise unused: a raw pool has no decoder)
+    c->raw_maps = g.storage == KVCAR_BF16;
+    for (int i = 0; i < nl * 2 && c->raw_maps; ++i) {
+        if (c->ae[i].set || c->width[i] == 0) continue;
+        c->raw_maps = raw_build_map(img.data() + c->tmap_off + (size_t)i * 3 * 128, c->pool + c->pool_off[i],
+                                    (size_t)g.max_pages * g.page_tokens, (uint64_t)c->width[i]);
+    }
     c->tc.pbuf = reinterpret_cast<float *>(c->ws + c->kvsplit_off);
     c->tc.pflags = reinterpret_cast<uint32_t *>(c->ws + c->kvsplit_off +
                                                 (size_t)TC_SPLIT_TILES * g.n_q_heads * 132 * sizeof(float));
@@ -786,6 +794,7 @@ static int prepare_decode(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int3
     a.max_chunks = c->max_chunks;
     a.flags = flags;
     a.scale = 1.0f / std::sqrt((float)g.head_dim);
+    a.raw_tmaps = c->raw_maps ? c->weights + c->tmap_off : nullptr;
     sl.n = n_seqs;
     memcpy(sl.id, seqs, (size_t)n_seqs * 4);
     return (max_len + c->chunk_tokens - 1) / c->chunk_tokens;

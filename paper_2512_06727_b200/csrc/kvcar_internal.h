@@ -81,6 +81,8 @@ struct DecodeArgs {
     int32_t chunk_tokens, max_chunks;
     uint32_t flags;
     float scale;
+    const void *raw_tmaps;  // TMA descriptors of the raw (layer, K|V) pools (descriptor of pool i at + i * 384 bytes),
+                            // or null: the raw-row kernel then stages its rows with cp.async
 };
 
 struct EncodeArgs {
@@ -112,6 +114,9 @@ cudaError_t launch_decode_generic(const DecodeArgs &a, const SeqList &seqs, int 
                                   int grid_chunks, cudaStream_t st);
 // raw K/V layers (no autoencoder), head_dim 64, <= 8 query heads per KV head (kvcar_raw.cu)
 cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtype, int grid_chunks, cudaStream_t st);
+// TMA descriptor of one raw bf16 pool [rows][width] with a box of 32 rows x 64 columns (one head's slice of one
+// 32-token step), 128-byte swizzle; false if the driver entry point is missing or the shape is refused
+bool raw_build_map(void *dst_host, const void *pool_dev, uint64_t rows, uint64_t width);
 // n_chunks: tiles of the longest listed sequence (picks the kernel: a warp or a CTA per sequence and query head)
 cudaError_t launch_combine(const DecodeArgs &a, const SeqList &seqs, int dtype, int n_chunks, cudaStream_t st);
 size_t decode_generic_smem(int hq, int hd, int max_d, int max_m);

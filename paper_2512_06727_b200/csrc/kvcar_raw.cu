@@ -12,7 +12,10 @@
 // loads and dots it with the group's pre-scaled queries (shared memory, broadcast reads).  Online softmax over
 // the tile's four 32-token groups (shuffle max / sum).  V phase: lane = channel pair; the warp reads one V row
 // per step, the row index and the probabilities come from the owning lane through shared memory.
+#include <cuda.h>
+
 #include "kvcar_internal.h"
+#include "kvcar_ptx.cuh"
 
 namespace kvcar {
 
@@ -62,10 +65,10 @@ struct Row64<float> {
 // where KV head h of this layer reads its rows: pool base, row width, first column
 struct HeadSrc {
     const void *pool;
-    int width, col;
+    int width, col, src_layer;
 };
 __device__ __forceinline__ HeadSrc find_head(const WhichPlan &wp, int h) {
-    HeadSrc r{nullptr, 0, 0};
+    HeadSrc r{nullptr, 0, 0, 0};
     for (int s = 0; s < wp.n_src; ++s) {
         const SourcePlan &sp = wp.src[s];
         for (int i = 0; i < sp.n_need; ++i)
@@ -73,6 +76,7 @@ __device__ __forceinline__ HeadSrc find_head(const WhichPlan &wp, int h) {
                 r.pool = sp.pool;
                 r.width = sp.width;
                 r.col = sp.slot[i] * 64;
+                r.src_layer = sp.src_layer;
             }
     }
     return r;
@@ -207,6 +211,11 @@ __global__ void __launch_bounds__(RW * 32, 4) decode_raw_kernel(const __grid_con
 // are; the probabilities come out in the layout the next product wants as its row operand (queries x tokens), and
 // V enters through transposing matrix loads.  Online softmax across the four 32-token steps, fp32.  Groups of
 // fewer than 8 heads leave the other operand rows zero.
+// TMA build: where a 32-token step lies inside one page (page size a multiple of 32) and the pools have tensor
+// maps, one elected lane fetches a step with two tensor loads (a 32-row x 64-column box of the K pool and of the V
+// pool, 128-byte swizzle: the same layout the cp.async build writes by hand) that count their bytes on a barrier
+// of the warp, instead of sixteen 16-byte copies and eight page-table look-ups per lane.  (Requesting
+// the whole tile at once - four buffers per warp - halves the resident warps and measured slower at every size.)
 constexpr int GQ_STEP = 32;                      // tokens per step
 constexpr int GQ_BUF = GQ_STEP * 64 * 2;         // bytes of one K (or V) step buffer: 32 rows x 128 B
 constexpr int GQ_WARP_SMEM = 4 * GQ_BUF;         // K and V, two steps each
@@ -241,9 +250,11 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
+template <bool TMA>
 __global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_constant__ DecodeArgs a,
                                                                const __grid_constant__ SeqList seqs) {
     extern __shared__ __align__(128) uint8_t gq_smem[];
+    __shared__ __align__(8) uint64_t step_bar[GQ_RW][2];  // TMA build: bytes of a step buffer pair have landed
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x, h = blockIdx.y * GQ_RW + warp, si = blockIdx.z;
     if (h >= a.hkv) return;
@@ -257,7 +268,23 @@ __global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_
     const __nv_bfloat16 *kpool = reinterpret_cast<const __nv_bfloat16 *>(ks.pool) + ks.col;
     const __nv_bfloat16 *vpool = reinterpret_cast<const __nv_bfloat16 *>(vs.pool) + vs.col;
     const int32_t *bt = a.block_table + (int64_t)seq * a.max_pages_per_seq;
-    const uint32_t sbase = smem_addr(gq_smem) + warp * GQ_WARP_SMEM;  // K step buffers 0, 1, then V step buffers 0, 1
+    // K step buffers 0, 1, then V step buffers 0, 1 (1024-byte aligned: the swizzle pattern of the tensor loads is a
+    // function of the address)
+    const uint32_t sbase = ((smem_addr(gq_smem) + 1023u) & ~1023u) + warp * GQ_WARP_SMEM;
+    uint8_t *gbase = gq_smem + (sbase - smem_addr(gq_smem));
+    const uint32_t bar0 = smem_addr(&step_bar[warp][0]);
+    const char *kmap = nullptr, *vmap = nullptr;
+    if (TMA) {
+        kmap = reinterpret_cast<const char *>(a.raw_tmaps) + (size_t)(ks.src_layer * 2) * 384;
+        vmap = reinterpret_cast<const char *>(a.raw_tmaps) + (size_t)(vs.src_layer * 2 + 1) * 384;
+        if (lane == 0) {
+            ptx::mbar_init(bar0, 1);
+            ptx::mbar_init(bar0 + 8, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        ptx::fence_async_smem();
+        __syncwarp();
+    }
     const int g = lane >> 2, t = lane & 3;
 
     // this lane's part of the row operand Q[16 x 64] (rows >= group are zero): per 16-channel step, channels
@@ -274,6 +301,16 @@ __global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_
     // fetch one 32-token step: lane = (row within a group of four, 16-byte chunk); rows past the tile's end re-read
     // the tile's first row (their probabilities are zero)
     auto fetch = [&](int step, int buf) {
+        if (TMA) {
+            if (ptx::elect_one()) {
+                const int tok = t0 + GQ_STEP * step;  // the step's 32 tokens lie in one page
+                const int row = bt[tok / a.page_tokens] * a.page_tokens + tok % a.page_tokens;
+                ptx::mbar_expect_tx(bar0 + 8 * buf, 2 * GQ_BUF);
+                ptx::tma_load_2d(sbase + buf * GQ_BUF, kmap, ks.col, row, bar0 + 8 * buf);
+                ptx::tma_load_2d(sbase + (2 + buf) * GQ_BUF, vmap, vs.col, row, bar0 + 8 * buf);
+            }
+            return;
+        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int r = 4 * i + (lane >> 3), c = lane & 7;
@@ -295,8 +332,32 @@ __global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_
     fetch(0, 0);
     for (int step = 0; step < n_steps; ++step) {
         const int buf = step & 1;
-        if (step + 1 < n_steps) {
-            fetch(step + 1, buf ^ 1);
+        if (step + 1 < n_steps) fetch(step + 1, buf ^ 1);
+        if (TMA) {
+            // bounded like every wait on a barrier in this library: on expiry a code goes to the status word and the
+            // warp carries on to its normal exit
+            uint32_t n = 0;
+            uint64_t t_start = 0;
+            while (!ptx::mbar_try(bar0 + 8 * buf, (uint32_t)(step >> 1) & 1u)) {
+                if ((++n & 255u) == 0) {
+                    const uint64_t now = ptx::global_ns();
+                    if (t_start == 0) t_start = now;
+                    if (now - t_start > 2000000000ull) {
+                        atomicCAS(a.status, 0, 0x501);
+                        break;
+                    }
+                }
+            }
+            // rows past the tile's end hold whatever the page holds: their probabilities are zero, but zero times a
+            // stray NaN is not, so they are cleared
+            const int r_end = valid - GQ_STEP * step;
+            if (r_end < GQ_STEP && lane >= r_end) {
+                uint4 *kr = reinterpret_cast<uint4 *>(gbase + buf * GQ_BUF + lane * 128);
+                uint4 *vr = reinterpret_cast<uint4 *>(gbase + (2 + buf) * GQ_BUF + lane * 128);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) kr[i] = vr[i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        } else if (step + 1 < n_steps) {
             cp_async_wait<1>();
         } else {
             cp_async_wait<0>();
@@ -375,19 +436,31 @@ __global__ void __launch_bounds__(GQ_RW * 32) decode_raw_gq_kernel(const __grid_
 
 }  // namespace
 
+bool raw_build_map(void *dst_host, const void *pool_dev, uint64_t rows, uint64_t width) {
+    static EncodeTiledFn fn = tensor_map_encoder();
+    if (!fn || width % 8 != 0) return false;
+    return encode_bf16_map(fn, dst_host, pool_dev, rows, width, width, GQ_STEP);
+}
+
 cudaError_t launch_decode_raw(const DecodeArgs &a, const SeqList &seqs, int dtype, int grid_chunks, cudaStream_t st) {
     dim3 grid(grid_chunks, (a.hkv + RW - 1) / RW, seqs.n);
     if (dtype == KVCAR_BF16) {
         static bool configured[64] = {};  // per device: the attribute belongs to the device's copy of the kernel
         int dev = 0;
         cudaGetDevice(&dev);
+        constexpr int smem = GQ_SMEM + 1024;  // + room to align the step buffers
         if (dev < 0 || dev >= 64 || !configured[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(decode_raw_gq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GQ_SMEM);
+            cudaError_t e = cudaFuncSetAttribute(decode_raw_gq_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(decode_raw_gq_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < 64) configured[dev] = true;
         }
         grid.y = (a.hkv + GQ_RW - 1) / GQ_RW;
-        decode_raw_gq_kernel<<<grid, GQ_RW * 32, GQ_SMEM, st>>>(a, seqs);
+        if (a.raw_tmaps && a.page_tokens % GQ_STEP == 0)
+            decode_raw_gq_kernel<true><<<grid, GQ_RW * 32, smem, st>>>(a, seqs);
+        else
+            decode_raw_gq_kernel<false><<<grid, GQ_RW * 32, smem, st>>>(a, seqs);
         return cudaGetLastError();
     }
     if (dtype == KVCAR_F32)
