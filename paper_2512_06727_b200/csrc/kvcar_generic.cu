@@ -453,32 +453,53 @@ __global__ void __launch_bounds__(32 * CB_WARPS) combine_kernel(const __grid_con
     __shared__ float red[CB_WARPS];
     __shared__ float accs[CB_WARPS][128];
 
-    float M = -INFINITY;
-    for (int ch = c; ch < n_chunks; ch += 32 * CB_WARPS) M = fmaxf(M, base[ch * stride]);
-    M = block_reduce(M, true, red);
-    float S = 0.f;
-    for (int ch = c; ch < n_chunks; ch += 32 * CB_WARPS) {
-        const float m = base[ch * stride], s = base[ch * stride + 1];
-        S += (m == -INFINITY) ? 0.f : s * expf(m - M);
-    }
-    S = block_reduce(S, false, red);
+    // One pass: warp w folds tiles w, w + CB_WARPS, ... into a running (maximum, sum, weighted values), the loads of eight
+    // tiles in flight at a time (they do not depend on one another; only the fold does), then the
+    // warps' results are folded in shared memory.
+    constexpr int U = 8;
+    float Mw = -INFINITY, Sw = 0.f;
     float av[4] = {0.f, 0.f, 0.f, 0.f};  // channels lane, lane + 32, lane + 64, lane + 96
-#pragma unroll 4
-    for (int ch = warp; ch < n_chunks; ch += CB_WARPS) {
-        const float *part = base + ch * stride;
-        const float m = part[0];
-        const float w = (m == -INFINITY) ? 0.f : expf(m - M);
+    for (int ch0 = warp; ch0 < n_chunks; ch0 += U * CB_WARPS) {
+        float m[U], s_[U], v[U][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (lane + 32 * j < hd) av[j] = fmaf(w, part[2 + lane + 32 * j], av[j]);
+        for (int u = 0; u < U; ++u) {
+            const int ch = ch0 + u * CB_WARPS;
+            const float *part = base + (int64_t)ch * stride;
+            const bool in = ch < n_chunks;
+            m[u] = in ? part[0] : -INFINITY;
+            s_[u] = in ? part[1] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[u][j] = (in && lane + 32 * j < hd) ? part[2 + lane + 32 * j] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (m[u] == -INFINITY) continue;  // an empty tile (or none)
+            const float Mn = fmaxf(Mw, m[u]);
+            const float cw = (Mw == -INFINITY) ? 0.f : expf(Mw - Mn), cn = expf(m[u] - Mn);
+            Sw = Sw * cw + s_[u] * cn;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) av[j] = av[j] * cw + v[u][j] * cn;
+            Mw = Mn;
+        }
+    }
+    __shared__ float wM[CB_WARPS], wS[CB_WARPS];
+    if (lane == 0) {
+        wM[warp] = Mw;
+        wS[warp] = Sw;
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) accs[warp][lane + 32 * j] = av[j];
     __syncthreads();
-    float acc = 0.f;
-    if (on)
+    float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < CB_WARPS; ++w) acc += accs[w][c];
+    for (int w = 0; w < CB_WARPS; ++w) M = fmaxf(M, wM[w]);
+    float S = 0.f, acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < CB_WARPS; ++w) {
+        const float f = (wM[w] == -INFINITY) ? 0.f : expf(wM[w] - M);
+        S += wS[w] * f;
+        if (on) acc += accs[w][c] * f;
+    }
 
     if (a.flags & KVCAR_INCLUDE_CURRENT_EXACT) {
         const int g = qh / (hq / a.hkv);
