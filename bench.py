@@ -806,6 +806,15 @@ def main():
                     row["raw_twin"] = {"tokens_per_s": u["tokens_per_s"], "us_per_launch": ru["avg_launch_us"],
                                        "bound": ru["bound"], "frac": ru["frac"], "achieved_gbs": ru["achieved"],
                                        "cache_bytes_per_token": u["cache_bytes_per_token"]}
+                # the headline workload once more with the K side in the absorbed form (same results up to rounding)
+                if wc.name == w.name and wc.storage == "bf16" and not args.absorbed and not args.uncompressed:
+                    class A2: pass
+                    a2 = A2(); a2.kernel = args.kernel; a2.absorbed = True
+                    ab = measure(wc, a2, torch, B, st_, 3, False, flush, peaks)
+                    ra = ab["roofline"]
+                    row["absorbed_k"] = {"tokens_per_s": ab["tokens_per_s"], "us_per_launch": ra["avg_launch_us"],
+                                         "frac_on_own_operation_count": ra["frac"],
+                                         "frac_if_credited_with_the_plain_form": ra.get("plain_form_equivalent_frac")}
             except Exception as ex:      # a configuration that does not fit or fails is reported, not fatal
                 row["error"] = str(ex)[:200]
             configs.append(row)

@@ -261,3 +261,21 @@ def test_reuse_map_from_l1_matches_oracle_bit_for_bit():
         B.head_l1_scratch_bytes(1, 12, 8192)                  # one layer has no layer below
     with pytest.raises(B.KvcarError):
         B.head_l1_distance(12, 12, 60, B.BF16, 16, 8, 16, 1 << 20, 16)   # a 60-wide head is not whole 16-byte chunks
+
+
+def test_trace_report_reads_synthetic_stamps(capsys):
+    """The time-stamp reader of the tensor kernel (python -m paper_2512_06727_b200.trace) on hand-made records: two
+    jobs of the issuer (a hidden chunk of two slabs, a head group of one) and their epilogues."""
+    from paper_2512_06727_b200 import trace
+    iss = [(100, 0x11), (150, 0x30), (400, 0x31), (500, 0x30), (800, 0x31), (900, 0x19),
+           (1000, 0x12), (1100, 0x30), (1400, 0x31), (1500, 0x19)]
+    ep = [(50, 0x40), (950, 0x41), (1950, 0x43), (2000, 0x50), (2100, 0x51), (2200, 0x52), (2600, 0x53)]
+    trace.report({"0.0": [], "0.1": [], "0.2": iss, "0.3": ep, "1.0": [], "1.1": [], "1.2": [], "1.3": []}, 5)
+    out = capsys.readouterr().out
+    assert "issuer: 2 jobs, 3 slabs in 1400 cycles; waiting 250, issuing 850, between jobs 100" in out
+    assert "hidden chunk jobs: 1, mean 800 cycles, 400 per slab" in out
+    assert "head group jobs: 1, mean 500 cycles, 500 per slab" in out
+    assert "epilogue, hidden chunk: 1 jobs, mean wait 900, mean work 1000 cycles" in out
+    trace.report({"0.2": [], "0.3": []}, 5)
+    assert "no stamps" in capsys.readouterr().out
+
