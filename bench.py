@@ -48,6 +48,8 @@ def parse():
     ap.add_argument("--absorbed", action="store_true",
                     help="pass KVCAR_ABSORBED: K scores from the hidden vectors (absorbed last decoder layer); the roofline "
                          "then counts that form's own, smaller number of operations")
+    ap.add_argument("--absorbed-v", action="store_true",
+                    help="with --absorbed: KVCAR_ABSORBED_V as well (the V side through the hidden vectors too)")
     ap.add_argument("--api", default="fused", choices=["fused", "split"],
                     help="a layer's step through kvcar_step_layer (one call; the tile kernel runs beside the encoder) "
                          "or through kvcar_encode_append + kvcar_decode_attention")
@@ -601,7 +603,8 @@ def measure(w, args, torch, B, steps, warmup, uncompressed, flush, peaks, fused=
     seqs = list(range(w.batch))
     stream = sess.stream()
     absorbed = bool(getattr(args, "absorbed", False)) and not uncompressed
-    flags = B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if absorbed else 0)
+    both = absorbed and bool(getattr(args, "absorbed_v", False))
+    flags = B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if absorbed else 0) | (B.ABSORBED_V if both else 0)
     n_in = 4
     k, v, q, out = step_inputs(sess, w, torch, n_in)       # a few input sets, cycled (values do not matter)
     for i in range(warmup):
@@ -638,12 +641,13 @@ def measure(w, args, torch, B, steps, warmup, uncompressed, flush, peaks, fused=
     torch.cuda.synchronize()
     sess.ctx.sync_status(stream)
     plain_flops = sum(sess.ctx.layer_work_per_token(l)[1] * L * w.batch for (l, L, _, _) in kev)
-    flops = sum(sess.ctx.layer_work_absorbed(l) * L * w.batch for (l, L, _, _) in kev) if absorbed else plain_flops
+    flops = sum(sess.ctx.layer_work_absorbed(l, both) * L * w.batch for (l, L, _, _) in kev) if absorbed else plain_flops
     byts = sum(sess.ctx.layer_work_per_token(l)[0] * L * w.batch for (l, L, _, _) in kev)
     kern_s = sum(a_.elapsed_time(b_) for (_, _, a_, b_) in kev) / 1e3
     roof = roofline_of(flops, byts, kern_s, peaks, len(kev))
     if absorbed:   # the plain form's operations over the same time: what the absorbed form is worth as plain-form throughput
-        roof["form"] = "absorbed K scores (KVCAR_ABSORBED): achieved and frac count this form's own operations"
+        roof["form"] = ("absorbed K and V sides (KVCAR_ABSORBED | KVCAR_ABSORBED_V)" if both else
+                        "absorbed K scores (KVCAR_ABSORBED)") + ": achieved and frac count this form's own operations"
         roof["plain_form_flops_per_launch"] = plain_flops / len(kev)
         roof["plain_form_equivalent_frac"] = plain_flops / kern_s / 1e12 / roof["peak"] if roof.get("bound") == "tensor" else None
     comp, full = sess.ctx.cache_bytes_per_token()
@@ -716,7 +720,8 @@ def main():
     sess, src, aes, k, v, q, out = head.pop("session")
     seqs = list(range(w.batch))
     stream = sess.stream()
-    flags = B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if (args.absorbed and not args.uncompressed) else 0)
+    flags = B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if (args.absorbed and not args.uncompressed) else 0) | \
+        (B.ABSORBED_V if (args.absorbed and args.absorbed_v and not args.uncompressed) else 0)
 
     # ---- e2e: host buffers through the C ABI, copies inside the timed region ----
     e2e = None
@@ -809,12 +814,13 @@ def main():
                 # the headline workload once more with the K side in the absorbed form (same results up to rounding)
                 if wc.name == w.name and wc.storage == "bf16" and not args.absorbed and not args.uncompressed:
                     class A2: pass
-                    a2 = A2(); a2.kernel = args.kernel; a2.absorbed = True
-                    ab = measure(wc, a2, torch, B, st_, 3, False, flush, peaks)
-                    ra = ab["roofline"]
-                    row["absorbed_k"] = {"tokens_per_s": ab["tokens_per_s"], "us_per_launch": ra["avg_launch_us"],
-                                         "frac_on_own_operation_count": ra["frac"],
-                                         "frac_if_credited_with_the_plain_form": ra.get("plain_form_equivalent_frac")}
+                    for key, both_ in (("absorbed_k", False), ("absorbed_kv", True)):
+                        a2 = A2(); a2.kernel = args.kernel; a2.absorbed = True; a2.absorbed_v = both_
+                        ab = measure(wc, a2, torch, B, st_, 3, False, flush, peaks)
+                        ra = ab["roofline"]
+                        row[key] = {"tokens_per_s": ab["tokens_per_s"], "us_per_launch": ra["avg_launch_us"],
+                                    "frac_on_own_operation_count": ra["frac"],
+                                    "frac_if_credited_with_the_plain_form": ra.get("plain_form_equivalent_frac")}
             except Exception as ex:      # a configuration that does not fit or fails is reported, not fatal
                 row["error"] = str(ex)[:200]
             configs.append(row)
@@ -827,7 +833,7 @@ def main():
                            "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
                            "latent_full": 0 if args.uncompressed else w.latent_full, "reuse_frac": w.reuse_frac,
                            "page_tokens": w.page_tokens, "kernel": args.kernel, "api": args.api,
-                           "uncompressed": bool(args.uncompressed), "absorbed": bool(args.absorbed and not args.uncompressed),
+                           "uncompressed": bool(args.uncompressed), "absorbed": ("kv" if args.absorbed_v else "k") if (args.absorbed and not args.uncompressed) else False,
                            "storage": w.storage,
                            "l2": "flushed between steps and between the per-launch timings (256 MiB write outside the event pairs)",
                            "cache_bytes_per_token": head["cache_bytes_per_token"],

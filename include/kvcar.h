@@ -64,6 +64,7 @@ typedef enum {
 /* flags of kvcar_decode_attention */
 #define KVCAR_INCLUDE_CURRENT_EXACT 1u /* also attend to the current token through its exact K/V */
 #define KVCAR_ABSORBED 2u /* K side through the absorbed last decoder layer (see kvcar_decode_attention) */
+#define KVCAR_ABSORBED_V 4u /* with KVCAR_ABSORBED: the V side too */
 
 #define KVCAR_MAX_BATCH 512    /* sequences per launching call   */
 #define KVCAR_MAX_KV_HEADS 32
@@ -215,7 +216,12 @@ kvcar_status kvcar_advance(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, 
  * never formed.  The same result up to rounding (W4_h^T q is rounded to the
  * storage type once per sequence and head); honoured by the tensor-core kernel
  * for K when the launch fills the machine, ignored (plain form computed) by
- * every other kernel and for V.
+ * every other kernel.  KVCAR_ABSORBED_V (only together with KVCAR_ABSORBED): the
+ * same for V, sum_t p_t v'_t = W4_h (sum_t p_t a_t) + b4_h sum_t p_t: a tile
+ * hands on sum_t p_t a_t (m values per query head) and the last layer is applied
+ * once per sequence and head when the tiles are merged; the probabilities enter
+ * that product rounded to the storage type.  For at most 16 query heads; ignored
+ * elsewhere.
  */
 kvcar_status kvcar_decode_attention(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                     const void *q, void *out, uint32_t flags, void *stream);
@@ -315,8 +321,10 @@ kvcar_status kvcar_layer_work_per_token(kvcar_ctx *ctx, int32_t layer, double *b
 /* The same count of floating-point operations for the KVCAR_ABSORBED form: on the K side the second decoder layer
  * (2 m 64 per needed head) and the 2 * 64 of q.k' per query head are replaced by 2 m per query head (the score taken
  * from the hidden vector); V side and bytes unchanged.  The per-sequence cost of W4_h^T q (m * 64 multiply-adds per
- * query head and call, not per token) is left out. */
-kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *ctx, int32_t layer, double *flops);
+ * query head and call, not per token) is left out.  both_sides != 0: the count for KVCAR_ABSORBED | KVCAR_ABSORBED_V,
+ * where the V side's second decoder layer and p.v' are likewise replaced by 2 m per query head (the per-sequence
+ * W4_h product of the merge left out). */
+kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *ctx, int32_t layer, int32_t both_sides, double *flops);
 /* Number of kernels the library has launched so far on this context. */
 kvcar_status kvcar_launch_count(kvcar_ctx *ctx, int64_t *count);
 /* Kernel family (kvcar_kernel: GENERIC, TENSOR or RAW) that kvcar_decode_attention will use

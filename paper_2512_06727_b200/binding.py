@@ -19,6 +19,7 @@ K, V = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TENSOR, KERNEL_RAW = 0, 1, 2, 3
 INCLUDE_CURRENT_EXACT = 1
 ABSORBED = 2
+ABSORBED_V = 4
 MAX_BATCH = 512
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "STATE", 3: "OOM_PAGES", 4: "WORKSPACE", 5: "UNSUPPORTED",
@@ -108,7 +109,7 @@ def _load(trace: bool = False) -> C.CDLL:
         "kvcar_pool_quant_layout": [vp, i32, i32, C.POINTER(sz)],
         "kvcar_cache_bytes_per_token": [vp, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "kvcar_layer_work_per_token": [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
-        "kvcar_layer_work_absorbed": [vp, i32, C.POINTER(C.c_double)],
+        "kvcar_layer_work_absorbed": [vp, i32, i32, C.POINTER(C.c_double)],
         "kvcar_launch_count": [vp, C.POINTER(C.c_int64)],
         "kvcar_layer_kernel": [vp, i32, ip],
         "kvcar_sync_status": [vp, vp],
@@ -316,9 +317,9 @@ class Context:
         self._check(self.lib.kvcar_layer_work_per_token(self._h, layer, C.byref(a), C.byref(b)))
         return a.value, b.value
 
-    def layer_work_absorbed(self, layer: int) -> float:
+    def layer_work_absorbed(self, layer: int, both_sides: bool = False) -> float:
         a = C.c_double()
-        self._check(self.lib.kvcar_layer_work_absorbed(self._h, layer, C.byref(a)))
+        self._check(self.lib.kvcar_layer_work_absorbed(self._h, layer, int(both_sides), C.byref(a)))
         return a.value
 
     def launch_count(self) -> int:

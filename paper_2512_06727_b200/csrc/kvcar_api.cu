@@ -202,7 +202,7 @@ void compute_layout(kvcar_ctx *c) {
         c->max_k_sources = std::max(c->max_k_sources, n);
     }
     c->abs_off = s;  // operands of the absorbed K scores (tensor-core kernel, KVCAR_ABSORBED)
-    s = align_up(s + tc_absorb_bytes(g, c->max_k_sources, c->max_m, nb), 256);
+    s = align_up(s + tc_absorb_bytes(g, c->max_k_sources, c->max_m, nb, c->max_chunks), 256);
     c->ws_bytes = s;
 }
 
@@ -546,7 +546,7 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
              (size_t)g.max_pages * g.page_tokens);
     {
         const size_t slot = c->tmap_off + (size_t)nl * 2 * 3 * 128;
-        tc_setup_absorb(c->tc, c->cfg, c->max_k_sources, c->max_m, std::min(g.max_seqs, KVCAR_MAX_BATCH),
+        tc_setup_absorb(c->tc, c->cfg, c->max_k_sources, c->max_m, std::min(g.max_seqs, KVCAR_MAX_BATCH), c->max_chunks,
                         c->ws + c->abs_off, img.data() + slot, c->weights + slot);
     }
     // descriptors of the raw pools (their three slots are otherwise unused: a raw pool has no decoder)
@@ -805,6 +805,7 @@ static int prepare_decode(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int3
 // step's encoder writes (the exact current token enters in the combine kernel).
 static kvcar_status enqueue_decode_tiles(kvcar_ctx *c, int32_t layer, const DecodeArgs &a, const SeqList &sl,
                                          int n_chunks, cudaStream_t st) {
+    c->tc.last_mode = 0;
     if (n_chunks <= 0) return KVCAR_OK;
     const kvcar_config &g = c->cfg;
     const bool want_tc = use_tensor_kernel(c) && tc_layer_supported(c->tc, layer);
@@ -830,7 +831,9 @@ static kvcar_status enqueue_decode_tiles(kvcar_ctx *c, int32_t layer, const Deco
 }
 
 static kvcar_status enqueue_combine(kvcar_ctx *c, const DecodeArgs &a, const SeqList &sl, int n_chunks, cudaStream_t st) {
-    cudaError_t e = launch_combine(a, sl, c->cfg.storage, n_chunks, st);
+    // a tile launch in the absorbed V form left U vectors, not weighted values: its own merge kernel reads them
+    cudaError_t e = c->tc.last_mode == 2 ? tc_launch_combine_absorbed(c->tc, a, sl, st)
+                                         : launch_combine(a, sl, c->cfg.storage, n_chunks, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "combine launch");
     ++c->launches;
     return KVCAR_OK;
@@ -843,7 +846,7 @@ static kvcar_status check_decode_args(kvcar_ctx *c, int32_t layer, const int32_t
         return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
     if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
-    if (flags & ~(KVCAR_INCLUDE_CURRENT_EXACT | KVCAR_ABSORBED)) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    if (flags & ~(KVCAR_INCLUDE_CURRENT_EXACT | KVCAR_ABSORBED | KVCAR_ABSORBED_V)) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
     return KVCAR_OK;
 }
 
@@ -1023,7 +1026,7 @@ kvcar_status kvcar_layer_work_per_token(kvcar_ctx *c, int32_t layer, double *byt
     return KVCAR_OK;
 }
 
-kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *c, int32_t layer, double *flops) {
+kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *c, int32_t layer, int32_t both_sides, double *flops) {
     if (!c || !flops || layer < 0 || layer >= c->cfg.n_layers) return fail(c, KVCAR_ERR_INVALID_ARG, "bad argument");
     const int hkv = c->cfg.n_kv_heads, hd = c->cfg.head_dim, group = c->cfg.n_q_heads / hkv;
     double f = 0;
@@ -1034,14 +1037,16 @@ kvcar_status kvcar_layer_work_absorbed(kvcar_ctx *c, int32_t layer, double *flop
             if (!need[s]) continue;
             const AEHost &a = c->ae[s * 2 + which];
             if (!a.set) {
-                if (which == 0) f += 2.0 * need[s] * group * hd;  // raw K rows: plain q.k
+                f += 2.0 * need[s] * group * hd;  // raw rows: plain q.k / p.v
                 continue;
             }
             f += 2.0 * a.latent * a.hidden;
-            f += which == 0 ? 2.0 * a.hidden * need[s] * group : 2.0 * a.hidden * hd * need[s];
+            if (which == 0 || both_sides)
+                f += 2.0 * a.hidden * need[s] * group;
+            else
+                f += 2.0 * a.hidden * hd * need[s] + 2.0 * need[s] * group * hd;  // second layer + p.v'
         }
     }
-    f += 2.0 * c->cfg.n_q_heads * hd;  // p.V
     *flops = f;
     return KVCAR_OK;
 }
@@ -1134,7 +1139,7 @@ extern "C" kvcar_status kvcar_decode_attention_static(kvcar_ctx *c, int32_t laye
         return fail(c, KVCAR_ERR_INVALID_ARG, "bad layer or pointer");
     if (!check_seqs(c, seqs, n_seqs)) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, KVCAR_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
-    if (flags & ~(KVCAR_INCLUDE_CURRENT_EXACT | KVCAR_ABSORBED)) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
+    if (flags & ~(KVCAR_INCLUDE_CURRENT_EXACT | KVCAR_ABSORBED | KVCAR_ABSORBED_V)) return fail(c, KVCAR_ERR_INVALID_ARG, "unknown flag");
     const kvcar_config &g = c->cfg;
     int max_len = 0;
     for (int i = 0; i < n_seqs; ++i) max_len = std::max(max_len, c->len[seqs[i]]);

@@ -94,6 +94,10 @@ struct PairLaunch {
     const void *tm_wq;  // TMA descriptor: box = 64 columns x nq_pad rows
     const float *qbias; // [source][abs_batch][nq_pad]
     int32_t nq_pad, abs_batch;
+    // absorbed V side (job kind 4): sum over a tile's tokens of p * a (a = activated hidden vector) per query head
+    float *ubuf;        // [listed sequence][tile][hq][m_pad_u]
+    int32_t m_pad_u;
+    uint32_t off_pop;   // shared-memory offset of the tile's probabilities as a bf16 column operand (0 = not this form)
 };
 
 // ---------------------------------------------------------------------------- waits
@@ -132,9 +136,11 @@ struct Bars {
     uint32_t p_ready;      // [1] both CTAs' probabilities of all K heads are in place (both CTAs)
     uint32_t s_free;       // [1] the peer's epilogue warps are done reading a pair's probabilities (both CTAs)
     uint32_t afull, aempty;  // [MAX_AUX] hidden slabs lent to the operand ring while they hold no activations
+    uint32_t pb_ready;       // [1] absorbed V: both CTAs' probability operands of the pair are written (leader)
+    uint32_t src_done;       // [1] absorbed V: every product that reads the current source's activations is complete
 };
 constexpr int MAX_AUX = 4 * MAX_HID_GROUPS;
-constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_AUX + 2 + 2 * MAX_AUX;
+constexpr uint32_t N_FIXED_BARS = 2 + 2 + MAX_AUX + 2 + 2 * MAX_AUX + 2;
 
 struct TileInfo {
     int si, chunk, valid;  // listed-sequence index, tile index inside the sequence, valid tokens (0 = no tile)
@@ -259,12 +265,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
     B.s_free = B.p_ready + 8;
     B.afull = B.s_free + 8;
     B.aempty = B.afull + 8 * MAX_AUX;
+    B.pb_ready = B.aempty + 8 * MAX_AUX;
+    B.src_done = B.pb_ready + 8;
 
     {  // this cluster's job tables -> shared memory
         const uint4 *src = reinterpret_cast<const uint4 *>(lay.parts + part_i);
         uint4 *dst = reinterpret_cast<uint4 *>(gbase + lay.off_part);
         for (int i = threadIdx.x; i < (int)(sizeof(TcPart) / 16); i += NTHREADS) dst[i] = src[i];
     }
+    if (lay.off_pop)  // the probability operand's padding rows are never written: they must hold finite values
+        for (int i = threadIdx.x; i < lay.nq_pad * 256 / 16; i += NTHREADS)
+            reinterpret_cast<uint4 *>(gbase + lay.off_pop)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int i = 0; i < lay.nslot; ++i) {
@@ -282,6 +293,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
             mbar_init(B.afull + 8 * i, 1);
             mbar_init(B.aempty + 8 * i, 1);
         }
+        mbar_init(B.pb_ready, 2 * N_EPI_WARPS);
+        mbar_init(B.src_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // tensor memory: all 512 columns in both CTAs of the pair (one CTA per SM by shared memory)
@@ -304,7 +317,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // places and wait for each of them to be free, so both see the same ring state.
         const uint32_t pid = warp == 0 ? 0u : 1u;
         if (elect_one()) {
-            uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0;
+            uint32_t slot = 0, phase = 0, aux_phase = 0, turn = 0, src_par = 0;
+            // Absorbed V launches: the job that reads a source's activations last stages nothing in the ring, so a free
+            // ring slot no longer proves that it is complete; the issuer signals src_done once per source instead and
+            // every producer waits for it once before it stages over the hidden slabs of the next source.
+            bool src_wait_due = false;
+            auto src_wait = [&]() {
+                mbar_wait(B.src_done, src_par ^ 1u, a.status, &abort_flag, 0x104);
+                src_par ^= 1u;
+                src_wait_due = false;
+            };
           for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride) {
             const TileInfo mine = locate_tile(tix, 2 * pair + (int)rank, seqs.n);
             TR(pid, 1);
@@ -345,6 +367,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         const int y0 = job.c0 + (int)rank * half_rows;
                         const int aux_lo = job.c0 >> 6, n_pool = lay.nslot + (ks_hid - aux_lo);
                         int r = 0;
+                        if (lay.off_pop && (job.first & 1)) src_wait_due = true;
                         // next staging place of this job: smem address in `dst`, leader's full barrier in `fb`
                         auto acquire1 = [&](uint32_t pair_bytes, bool own, uint32_t &dst, uint32_t &fb) {
                             if (r < lay.nslot) {
@@ -353,6 +376,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 fb = map_to_cta(B.full + 8 * sl, 0);
                             } else {
                                 const uint32_t x = (uint32_t)(aux_lo + r - lay.nslot);
+                                if (src_wait_due) src_wait();
                                 mbar_wait(B.aempty + 8 * x, ((aux_phase >> x) & 1u) ^ 1u, a.status, &abort_flag, 0x103);
                                 if (own && leader) mbar_expect_tx(B.afull + 8 * x, pair_bytes);
                                 aux_phase ^= 1u << x;
@@ -379,6 +403,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             }
                             TR(pid, 2);
                         }
+                        if (src_wait_due) src_wait();  // no lent slab was visited: the wait is owed once per source
+                    } else if (job.kind == 4) {
+                        // absorbed V: both operands are already in shared memory (activations, probabilities)
                     } else if (job.kind == 3) {
                         // absorbed scores: the column operand is this tile's sequence's W4_h^T q rows (all query heads)
                         const int ks2 = (sp.m + 63) >> 6;
@@ -433,7 +460,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         // and keeps descriptors and barrier addresses in uniform registers).
         if (leader && elect_one()) {
             constexpr bool issuer = true;
-            uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0;
+            uint32_t slot = 0, phase = 0, jc = 0, hid_phase = 0, aux_phase = 0, pair_it = 0;
             const int ks_hid = (lay.max_m + 63) >> 6;
             auto wait_full = [&]() -> uint32_t {
                 mbar_wait(B.full + 8 * slot, phase, a.status, &abort_flag, 0x201);
@@ -441,7 +468,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                 if (++slot == (uint32_t)lay.nslot) { slot = 0; phase ^= 1u; }
                 return s;
             };
-          for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride) {
+          for (int pair = pair0; pair < lay.n_pairs; pair += pair_stride, ++pair_it) {
+            bool pb_seen = false;
             for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
                 const int nj = P.n_jobs[which];
@@ -487,6 +515,47 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             }
                             TR(2, 0x31);
                         }
+                    } else if (job.kind == 4) {
+                        // absorbed V: U[feature][query] = sum over the tile's tokens of a[token][feature] * p[query][token].
+                        // Row operand = the hidden slabs read feature-major (each holds [token][64 features], i.e. an
+                        // MN-major tile: 64-feature atoms SLOT_BYTES apart, 8-token groups 1 KB apart); column operand =
+                        // this CTA's probabilities [query][token] in two 64-token atoms.  Each CTA supplies its own
+                        // tile's activations and probabilities, so its accumulator's own column block is its tile's U;
+                        // 128 features per product and CTA, all feature chunks side by side in one accumulator buffer
+                        // (an odd slab count repeats the second-to-last slab in the last chunk).
+                        const int ks2 = (m + 63) >> 6;
+                        constexpr bool slabwise = SLAB;
+                        for (int ks = 0; ks < ks2; ++ks)
+                            if (slabwise || (ks & 3) == 0) {
+                                const int ws = slabwise ? ks : min(ks + 3, ks2 - 1);
+                                mbar_wait(B.hid_ready + 8 * ws, (hid_phase >> ws) & 1u, a.status, &abort_flag, 0x204);
+                                hid_phase ^= 1u << ws;
+                            }
+                        if (!pb_seen) {
+                            mbar_wait(B.pb_ready, pair_it & 1u, a.status, &abort_flag, 0x207);
+                            pb_seen = true;
+                        }
+                        tc_fence_after();
+                        TR(2, 0x30);
+                        const uint32_t idesc = make_idesc(256, 2 * lay.nq_pad) | (1u << 15);  // row operand MN-major
+                        const uint32_t s_pop = base + lay.off_pop;
+                        const int n_ch = (ks2 + 1) >> 1;
+                        for (int c = 0; c < n_ch; ++c) {
+                            const int sa = min(2 * c, ks2 - 2);
+                            uint64_t da = make_desc(s_hidden + sa * SLOT_BYTES);
+                            da = (da & ~((uint64_t)0x3FFF << 16)) | ((uint64_t)(SLOT_BYTES >> 4) << 16);  // leading (feature-atom) stride
+                            const uint32_t acc_c = acc + (uint32_t)(c * 2 * lay.nq_pad);
+#pragma unroll
+                            for (int t = 0; t < TILE / 16; ++t) {
+                                const uint64_t a_t = da + (uint64_t)(t * (16 * 128 >> 4));
+                                const uint64_t b_t = make_desc(s_pop + (uint32_t)((t >> 2) * lay.nq_pad * 128)) + (uint64_t)((t & 3) * 2);
+                                if (t == 0)
+                                    umma_pair<0>(acc_c, a_t, b_t, idesc);
+                                else
+                                    umma_pair<1>(acc_c, a_t, b_t, idesc);
+                            }
+                        }
+                        TR(2, 0x31);
                     } else if (job.kind == 3) {
                         // absorbed scores: the whole job's column operand is a few KB, so several K slabs share a place
                         // and a barrier round; the waits for the activations are those of a first head group
@@ -518,7 +587,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     } else {
                         const int ks2 = (m + 63) >> 6;
                         const uint32_t idesc = which == 0 ? make_idesc(256, 64 * job.nh) : make_idesc(256, 256);
-                        const bool first_use = job.first != 0;  // first head group of this source
+                        const bool first_use = (job.first & 1) != 0;  // first head group of this source
                         constexpr bool slabwise = SLAB;
                         for (int ks = 0; ks < ks2; ++ks) {
                             if (first_use) {
@@ -548,6 +617,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         }
                     }
                     if (issuer) umma_commit_pair(B.jfull + 8 * buf);
+                    // absorbed V launches: last job of its source - its completion frees the hidden slabs for staging
+                    if (lay.off_pop && (job.first & 2)) umma_commit_pair(B.src_done);
                     TR(2, 0x19);
                 }
             }
@@ -634,6 +705,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
         for (int which = 0; which < 2; ++which) {  // constant trip count: `which` folds into the code below
                 if (which < which_lo || which >= which_hi) continue;
             const int nj = P.n_jobs[which];
+            if (which == 1 && lay.off_pop) {
+                // absorbed V: this warp's rows of the probability operand are written; the products read them
+                // through the asynchronous proxy
+                fence_async_smem();
+                __syncwarp();
+                if (elect_one()) mbar_arrive_remote(map_to_cta(B.pb_ready, 0));
+            }
             if (which == 1 && !lay.kv_split) {
                 if (GMMA) {
                     // this warp's probabilities are in place here; the peer's arrive as counted bytes, announced by one warp
@@ -668,7 +746,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                     b2 = s1 + 2 * m_pad;
                 }
                 if (job.kind == 1) {
-                    if (job.first && (!SLAB || it == 0)) {
+                    if ((job.first & 1) && (!SLAB || it == 0)) {
                         // this source's parameters: fetched into registers first, so that the global-memory
                         // latency overlaps the wait for the other warps
                         float ps[MAX_HID_GROUPS], pt[MAX_HID_GROUPS], pb[MAX_HID_GROUPS];
@@ -995,6 +1073,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                 if (ql < 0) continue;
                                 const int qh = h_lo * group + ql;
                                 float *srow = Smine + ql * PSTRIDE;
+                                if (lay.off_pop) {
+                                    // absorbed V: this tile's probabilities as the column operand of the U product:
+                                    // [query][token] bf16, two 64-token atoms of 128-byte rows, 128-byte swizzle
+                                    uint8_t *dst = gbase + lay.off_pop + (lane >> 4) * (lay.nq_pad * 128) + ql * 128 +
+                                                   ((((lane & 15) >> 1) ^ (ql & 7)) << 4) + 8 * (lane & 1);
+                                    *reinterpret_cast<uint2 *>(dst) =
+                                        make_uint2(pack_bf16(sc[u].x, sc[u].y), pack_bf16(sc[u].z, sc[u].w));
+                                }
                                 if (lay.kv_split) {
                                     float *grow = lay.pbuf + ((size_t)(2 * pair + (int)rank) * hq + qh) * PSTRIDE;
                                     *reinterpret_cast<float4 *>(grow + 4 * lane) = sc[u];
@@ -1045,6 +1131,34 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                          : "memory");
                     }
                     TR(3, 0x53);
+                } else if (job.kind == 4) {
+                    // absorbed V: this thread owns hidden feature `row` of each 128-feature chunk; the accumulator's
+                    // own column block holds U[feature][query] of this CTA's tile; it goes to the workspace as it is
+                    // (the last decoder layer is applied once per sequence and head, after the tiles are merged)
+                    const uint32_t mask = (uint32_t)job.c0 | ((uint32_t)job.nc << 16);
+                    const int ks2 = (m + 63) >> 6, n_ch = (ks2 + 1) >> 1;
+                    if (mine.valid > 0) {
+                        float *ub = lay.ubuf + (((int64_t)mine.si * a.max_chunks + mine.chunk) * hq) * lay.m_pad_u;
+                        for (int c = chalf; c < n_ch; c += 2) {
+                            const int sa = min(2 * c, ks2 - 2);
+                            const int f = sa * 64 + row;
+                            const bool repeated = 2 * c > ks2 - 2 && row < 64;  // slab already covered by the chunk before
+                            float u[16];
+                            const uint32_t ta = acc + (uint32_t)(c * 2 * lay.nq_pad + lay.nq_pad * (int)rank);
+                            tmem_ld8(ta, u);
+                            tmem_ld8(ta + 8u, u + 8);
+                            tmem_ld_wait();
+                            if (!repeated && f < m) {
+#pragma unroll
+                                for (int ql = 0; ql < 16; ++ql)
+                                    if ((mask >> ql) & 1u) ub[(int64_t)ql * lay.m_pad_u + f] = u[ql];
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (elect_one()) mbar_arrive_remote(jempty_leader[buf]);
+                    TR(3, 0x63);
                 } else {
                     // V: this thread owns (head place, channel) = row; columns = tokens of tile chalf
                     if (!lay.kv_split && !p_waited) {
@@ -1184,7 +1298,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 // ---------------------------------------------------------------------------- host side
 inline uint32_t up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslots, int nslot) {
+PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslots, int nslot, bool pop = false) {
     PairLaunch l{};
     const int ks_hid = (max_m + 63) / 64;
     uint32_t o = 0;
@@ -1205,6 +1319,11 @@ PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslot
     if (l.group_mma) o = up(o + (uint32_t)nq_local * QBS * 2, 16);
     l.off_pb = o;
     if (l.group_mma) o = up(o + 2u * (uint32_t)nq_local * PBS * 2, 16);
+    if (pop) {  // absorbed V: the tile's probabilities as a column operand, 16 rows x 256 B, on a swizzle boundary
+        o = up(o, 1024);
+        l.off_pop = o;
+        o += 16 * 256;
+    }
     l.off_bar = o;
     l.nslot = nslot;
     l.max_m = max_m;
@@ -1215,16 +1334,16 @@ PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslot
 uint32_t launch_bytes(const PairLaunch &l) { return l.off_bar + 8u * (2 * l.nslot + N_FIXED_BARS) + 1024u; }
 
 // ring depth that fits beside everything else (0 = does not fit)
-int pick_nslot(int nq_local, int group, int max_m, int max_in, int pslots) {
+int pick_nslot(int nq_local, int group, int max_m, int max_in, int pslots, bool pop = false) {
     for (int nslot = 10; nslot >= 3; --nslot)
-        if (launch_bytes(make_launch(nq_local, group, max_m, max_in, pslots, nslot)) <= 227u * 1024u) return nslot;
+        if (launch_bytes(make_launch(nq_local, group, max_m, max_in, pslots, nslot, pop)) <= 227u * 1024u) return nslot;
     return 0;
 }
 
 // Job tables of one head subset [h_lo, h_hi) of one layer.  Returns false if it does not fit the table limits.
 // absorbed: the K head groups of every source are replaced by one score job over all its query heads (kind 3).
 bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int h_hi, TcPart &out, bool absorbed = false,
-                int group = 1) {
+                int group = 1, bool absorbed_v = false) {
     memset(&out, 0, sizeof(out));
     out.h_lo = h_lo;
     out.h_hi = h_hi;
@@ -1273,6 +1392,22 @@ bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int
                 out.abs_n[ns] = (uint8_t)cnt;
                 n = 0;  // no head groups
             }
+            if (absorbed_v && which == 1) {
+                // one job for the whole source: at most 16 query heads, at least two hidden slabs (the row operand
+                // spans two), and all 128-feature chunks side by side in one 256-column accumulator buffer
+                const int ks2 = (sp.m + 63) / 64;
+                if (nj == TC_MAX_JOBS || (h_hi - h_lo) * group > 16 || ks2 < 2 || ((ks2 + 1) / 2) * 32 > 256) return false;
+                TcJob &jb = out.jobs[which][nj++];
+                jb.kind = 4;
+                jb.src = (uint8_t)ns;
+                jb.first = 1;
+                uint32_t mask = 0;
+                for (int i = 0; i < n; ++i)
+                    for (int g = 0; g < group; ++g) mask |= 1u << ((heads[i] - h_lo) * group + g);
+                jb.c0 = (uint16_t)(mask & 0xffffu);
+                jb.nc = (uint16_t)(mask >> 16);
+                n = 0;
+            }
             for (int i = 0; i < n;) {  // head groups: K 4/2/1 real heads; V always four places, padded
                 if (nj == TC_MAX_JOBS) return false;
                 TcJob &jb = out.jobs[which][nj++];
@@ -1295,6 +1430,7 @@ bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int
                 }
                 i += nh;
             }
+            if (absorbed_v) out.jobs[which][nj - 1].first |= 2;  // last job of its source: its completion is signalled
             ++ns;
         }
         out.n_src[which] = ns;
@@ -1374,17 +1510,127 @@ __global__ void __launch_bounds__(128) absorb_q_kernel(const __grid_constant__ D
     }
 }
 
-size_t tc_absorb_bytes(const kvcar_config &cfg, int max_k_sources, int max_m, int batch) {
+// Merge of the tiles after a launch in the absorbed V form.  A tile's partial is (maximum, sum) in the usual place
+// and U = sum over its tokens of p * a (m values) in the U buffer; with w_t = exp(max_t - M) the head's output is
+// (W4_h (sum_t w_t U_t) + b4_h sum_t w_t s_t [+ the exact current token]) / (sum of all weights): the last decoder
+// layer is applied once, here.  One block per (query head, listed sequence); W4 is read through its transposed copy
+// [m][in_dim] so that consecutive threads read consecutive channels.
+constexpr int CA_THREADS = 128, CA_MAX_TILES = 512;
+__global__ void __launch_bounds__(CA_THREADS) combine_absorbed_kernel(const __grid_constant__ DecodeArgs a,
+                                                                      const __grid_constant__ SeqList seqs,
+                                                                      const float *ubuf, int m_pad) {
+    extern __shared__ float ca_smem[];  // U accumulated over the tiles [m_pad]
+    __shared__ float wts[CA_MAX_TILES];
+    __shared__ float red[CA_THREADS / 32];
+    const int qh = blockIdx.x, si = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int seq = seqs.id[si];
+    const int L = a.seq_len[seq];
+    const int hq = a.hq, hd = 64;
+    const int n_tiles = (L + a.chunk_tokens - 1) / a.chunk_tokens;
+    const int kvh = qh / (hq / a.hkv);
+    const WhichPlan &wp = a.plan->w[1];
+    int s_ = 0, slot = 0;
+    for (int i = 0; i < wp.n_src; ++i)
+        for (int k = 0; k < wp.src[i].n_need; ++k)
+            if (wp.src[i].kv_head[k] == kvh) {
+                s_ = i;
+                slot = wp.src[i].slot[k];
+            }
+    const SourcePlan &sp = wp.src[s_];
+    const float *part = a.partials + ((int64_t)si * a.max_chunks * hq + qh) * (hd + 2);
+    const int64_t pstride = (int64_t)hq * (hd + 2);
+    auto block_max = [&](float v) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+        __syncthreads();
+        if (lane == 0) red[warp] = v;
+        __syncthreads();
+        float r = red[0];
+#pragma unroll
+        for (int i = 1; i < CA_THREADS / 32; ++i) r = fmaxf(r, red[i]);
+        return r;
+    };
+    auto block_sum = [&](float v) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        __syncthreads();
+        if (lane == 0) red[warp] = v;
+        __syncthreads();
+        float r = red[0];
+#pragma unroll
+        for (int i = 1; i < CA_THREADS / 32; ++i) r += red[i];
+        return r;
+    };
+    float M = -INFINITY;
+    for (int t = tid; t < n_tiles; t += CA_THREADS) M = fmaxf(M, part[t * pstride]);
+    M = block_max(M);
+    float S = 0.f;
+    for (int t = tid; t < n_tiles; t += CA_THREADS) {
+        const float mt = part[t * pstride];
+        const float w = mt == -INFINITY ? 0.f : expf(mt - M);
+        wts[t] = w;
+        S += w * part[t * pstride + 1];
+    }
+    S = block_sum(S);  // (the barriers inside also publish wts)
+    const float *ub = ubuf + (((int64_t)si * a.max_chunks) * hq + qh) * m_pad;
+    const int64_t ustride = (int64_t)hq * m_pad;
+    for (int j = tid; j < sp.m; j += CA_THREADS) {
+        float acc = 0.f;
+#pragma unroll 4
+        for (int t = 0; t < n_tiles; ++t) acc = fmaf(wts[t], ub[t * ustride + j], acc);
+        ca_smem[j] = acc;
+    }
+    __syncthreads();
+    // channel c of the head: two threads split the hidden range
+    const int c = tid & 63, half = tid >> 6;
+    const __nv_bfloat16 *w2t = reinterpret_cast<const __nv_bfloat16 *>(sp.w2t) + slot * hd + c;
+    float o = 0.f;
+    for (int j = half; j < sp.m; j += 2) o = fmaf(__bfloat162float(w2t[(int64_t)j * sp.in_dim]), ca_smem[j], o);
+    __shared__ float o2[64];
+    if (half == 1) o2[c] = o;
+    __syncthreads();
+    float acc = half == 0 ? o + o2[c] + sp.b2[slot * hd + c] * S : 0.f;
+    if (a.flags & KVCAR_INCLUDE_CURRENT_EXACT) {
+        const int W = a.hkv * hd;
+        const __nv_bfloat16 *kc = reinterpret_cast<const __nv_bfloat16 *>(a.plan->cur[0][kvh]) + (int64_t)seq * W + a.plan->cur_head[0][kvh] * hd;
+        const __nv_bfloat16 *vc = reinterpret_cast<const __nv_bfloat16 *>(a.plan->cur[1][kvh]) + (int64_t)seq * W + a.plan->cur_head[1][kvh] * hd;
+        const __nv_bfloat16 *qg = reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((int64_t)si * hq + qh) * hd;
+        const float sc = block_sum(half == 0 ? __bfloat162float(qg[c]) * __bfloat162float(kc[c]) : 0.f) * a.scale;
+        const float Mn = fmaxf(M, sc);
+        const float c0 = M == -INFINITY ? 0.f : expf(M - Mn), c1 = expf(sc - Mn);
+        S = S * c0 + c1;
+        acc = acc * c0 + __bfloat162float(vc[c]) * c1;
+    }
+    if (half == 0)
+        reinterpret_cast<__nv_bfloat16 *>(a.out)[((int64_t)si * hq + qh) * hd + c] = __float2bfloat16_rn(S > 0.f ? acc / S : 0.f);
+}
+
+cudaError_t tc_launch_combine_absorbed(const TcState &tc, const DecodeArgs &a, const SeqList &seqs, cudaStream_t st) {
+    combine_absorbed_kernel<<<dim3(a.hq, seqs.n), CA_THREADS, (size_t)tc.abs_m_pad * sizeof(float), st>>>(a, seqs, tc.ubuf,
+                                                                                                        tc.abs_m_pad);
+    return cudaGetLastError();
+}
+
+// absorbed V side: bytes of the U vectors (0 where the form is not taken: more than 16 query heads, or more than
+// 512 tiles per sequence, which the merge kernel's weight table does not hold)
+static size_t absorb_u_bytes(const kvcar_config &cfg, int max_m, int batch, int max_chunks) {
+    if (cfg.n_q_heads > 16 || max_chunks > 512) return 0;
+    const size_t m_pad = ((size_t)max_m + 63) / 64 * 64;
+    return (size_t)batch * max_chunks * cfg.n_q_heads * m_pad * sizeof(float);
+}
+size_t tc_absorb_bytes(const kvcar_config &cfg, int max_k_sources, int max_m, int batch, int max_chunks) {
     if (cfg.storage != KVCAR_BF16 || cfg.n_q_heads > TC_ABS_MAX_Q || max_k_sources <= 0 || max_m <= 0) return 0;
     const size_t nq_pad = cfg.n_q_heads <= 16 ? 16 : 32, m_pad = ((size_t)max_m + 63) / 64 * 64;
     const size_t rows = (size_t)max_k_sources * batch * nq_pad;
-    return (rows * m_pad * 2 + 255) / 256 * 256 + rows * sizeof(float);
+    return (rows * m_pad * 2 + 255) / 256 * 256 + (rows * sizeof(float) + 255) / 256 * 256 +
+           absorb_u_bytes(cfg, max_m, batch, max_chunks);
 }
 
-void tc_setup_absorb(TcState &tc, const kvcar_config &cfg, int max_k_sources, int max_m, int batch, char *ws_area,
-                     char *tmap_host, char *tmap_dev) {
+void tc_setup_absorb(TcState &tc, const kvcar_config &cfg, int max_k_sources, int max_m, int batch, int max_chunks,
+                     char *ws_area, char *tmap_host, char *tmap_dev) {
     tc.wq = nullptr;
-    if (!tc.available || tc_absorb_bytes(cfg, max_k_sources, max_m, batch) == 0) return;
+    tc.ubuf = nullptr;
+    if (!tc.available || tc_absorb_bytes(cfg, max_k_sources, max_m, batch, max_chunks) == 0) return;
     EncodeTiledFn fn = tensor_map_encoder();
     if (!fn) return;
     const int nq_pad = cfg.n_q_heads <= 16 ? 16 : 32, m_pad = (max_m + 63) / 64 * 64;
@@ -1397,6 +1643,10 @@ void tc_setup_absorb(TcState &tc, const kvcar_config &cfg, int max_k_sources, in
     tc.abs_m_pad = m_pad;
     tc.abs_batch = batch;
     tc.abs_max_src = max_k_sources;
+    if (absorb_u_bytes(cfg, max_m, batch, max_chunks)) {
+        tc.ubuf = reinterpret_cast<float *>(ws_area + (rows * m_pad * 2 + 255) / 256 * 256 + (rows * sizeof(float) + 255) / 256 * 256);
+        tc.abs_max_chunks = max_chunks;
+    }
 }
 
 size_t tc_part_bytes(int n_layers) { return (size_t)n_layers * TC_PARTS_PER_LAYER * sizeof(TcPart); }
@@ -1489,8 +1739,10 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
             lc.split_ok[si] = fits ? 1 : 0;
         }
         if (!lc.split_ok[0]) continue;
-        lc.abs_ok = cfg.n_q_heads <= TC_ABS_MAX_Q &&
-                    build_part(plans[l], srcs, 0, cfg.n_kv_heads, parts[TC_PARTS_PER_LAYER - 1], true, group) ? 1 : 0;
+        lc.abs_ok = cfg.n_q_heads <= TC_ABS_MAX_Q && build_part(plans[l], srcs, 0, cfg.n_kv_heads, parts[7], true, group) ? 1 : 0;
+        lc.absv_ok = lc.abs_ok && cfg.n_q_heads <= 16 &&
+                     pick_nslot(cfg.n_kv_heads * group, group, max_m, max_in, pslots, true) >= 3 &&
+                     build_part(plans[l], srcs, 0, cfg.n_kv_heads, parts[8], true, group, true) ? 1 : 0;
         lc.ok = 1;
         lc.max_m = (uint16_t)max_m;
         lc.max_in = (uint16_t)max_in;
@@ -1545,8 +1797,12 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     }
     const int group = a.hq / a.hkv;
     const int nq_local = a.hkv / split * group;
+    // the absorbed forms: only where one cluster takes a pair's whole layer (no head or K/V split)
+    const bool absorbed = (a.flags & KVCAR_ABSORBED) && lc.abs_ok && tc.wq && split == 1 && !kv_split && seqs.n <= tc.abs_batch;
+    const bool absorbed_v = absorbed && (a.flags & KVCAR_ABSORBED_V) && lc.absv_ok && tc.ubuf && a.max_chunks <= tc.abs_max_chunks;
+    tc.last_mode = absorbed_v ? 2 : absorbed ? 1 : 0;
     PairLaunch lay = make_launch(nq_local, group, lc.max_m, lc.max_in, lc.pslots,
-                                 pick_nslot(nq_local, group, lc.max_m, lc.max_in, lc.pslots));
+                                 pick_nslot(nq_local, group, lc.max_m, lc.max_in, lc.pslots, absorbed_v), absorbed_v);
     lay.split = split;
     lay.n_pairs = n_pairs;
     lay.kv_split = kv_split;
@@ -1554,14 +1810,15 @@ cudaError_t tc_launch_decode(TcState &tc, const DecodeArgs &a, const SeqList &se
     lay.pbuf = tc.pbuf;
     lay.pflags = tc.pflags;
     lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * TC_PARTS_PER_LAYER + part_index(split, 0);
-    // the absorbed K form: only where one cluster takes a pair's whole layer (no head or K/V split)
-    if ((a.flags & KVCAR_ABSORBED) && lc.abs_ok && tc.wq && split == 1 && !kv_split && seqs.n <= tc.abs_batch) {
+    if (absorbed) {
         absorb_q_kernel<<<dim3(a.hq, seqs.n), 128, 0, st>>>(a, seqs, reinterpret_cast<__nv_bfloat16 *>(tc.wq), tc.qbias,
                                                             tc.abs_nq_pad, tc.abs_m_pad, tc.abs_batch);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         *n_launches = 2;
-        lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * TC_PARTS_PER_LAYER + TC_PARTS_PER_LAYER - 1;
+        lay.parts = reinterpret_cast<const TcPart *>(tc.parts_dev) + (size_t)layer * TC_PARTS_PER_LAYER + (absorbed_v ? 8 : 7);
+        lay.ubuf = tc.ubuf;
+        lay.m_pad_u = tc.abs_m_pad;
         lay.tm_wq = tc.tm_wq;
         lay.qbias = tc.qbias;
         lay.nq_pad = tc.abs_nq_pad;

@@ -8,7 +8,8 @@ constexpr int TC_MAX_LAYERS = 512;
 constexpr int TC_MAX_SRC = 6;    // distinct source layers per K or V of one head subset
 constexpr int TC_MAX_JOBS = 24;  // accumulator jobs per K or V of one head subset
 constexpr int TC_SPLIT_TILES = 160;  // the K/V split is used only while 2 x tiles <= SM count
-constexpr int TC_PARTS_PER_LAYER = 8;  // head subsets: whole, halves, quarters; then the whole with absorbed K scores
+constexpr int TC_PARTS_PER_LAYER = 9;  // head subsets: whole, halves, quarters; then the whole with absorbed K scores,
+                                       // then the whole with absorbed K scores and the absorbed V side
 constexpr int TC_ABS_MAX_Q = 32;       // query heads the absorbed score job takes (two CTAs x 32 columns at most)
 
 // One source layer as the tensor-core kernel sees it.
@@ -24,8 +25,9 @@ struct TcSrc {
 // up to four restored heads (second decoder layer).  The TMA producer, the MMA issuer
 // and the epilogue warps all walk the same list in the same order.
 struct TcJob {
-    uint8_t kind;    // 1 = hidden chunk, 2 = head group, 3 = absorbed scores of all query heads of the source (K only;
-                     // c0 | nc << 16 is then the mask of the source's local query heads)
+    uint8_t kind;    // 1 = hidden chunk, 2 = head group, 3 = absorbed scores of all query heads of the source (K only),
+                     // 4 = absorbed V side: sum over the tile's tokens of p * hidden vector for all query heads of
+                     // the source (for 3 and 4, c0 | nc << 16 is the mask of the source's local query heads)
     uint8_t src;     // index into TcPart::src[which]
     uint8_t nh;      // head group: real heads (1..4)
     uint8_t first;   // first job of its source
@@ -54,6 +56,7 @@ struct TcLayerCfg {
     uint16_t max_in;       // widest restored row among the layer's sources
     uint16_t pslots;       // parameter blocks kept in shared memory (one per source if every hidden layer is one chunk)
     uint8_t abs_ok;        // the absorbed table (index 7) exists
+    uint8_t absv_ok;       // the table with the absorbed V side as well (index 8) exists
 };
 
 struct TcState {
@@ -65,6 +68,11 @@ struct TcState {
     float *qbias = nullptr;         // [max K sources][batch][nq_pad]
     const void *tm_wq = nullptr;    // TMA descriptor of wq (device memory), box = 64 columns x nq_pad rows
     int abs_nq_pad = 0, abs_m_pad = 0, abs_batch = 0, abs_max_src = 0;
+    // absorbed V side: per (listed sequence, tile, query head) the m-vector sum_t p_t a_t (workspace), and which form
+    // the last tile launch took (0 plain, 1 absorbed K, 2 absorbed K and V): the merge kernel has to match it
+    float *ubuf = nullptr;
+    int abs_max_chunks = 0;
+    int last_mode = 0;
     int n_sms = 148;
     // K/V split of small grids: probabilities cross from the K cluster to the V cluster through these
     float *pbuf = nullptr;       // [TC_SPLIT_TILES][n_q_heads][132]
@@ -78,10 +86,12 @@ size_t tc_part_bytes(int n_layers);
 // bytes of the probability hand-over area (pbuf then pflags) inside the workspace
 size_t tc_split_bytes(const kvcar_config &cfg);
 // bytes of the absorbed-score operands inside the workspace (0 if the shape does not take the absorbed form)
-size_t tc_absorb_bytes(const kvcar_config &cfg, int max_k_sources, int max_m, int batch);
+size_t tc_absorb_bytes(const kvcar_config &cfg, int max_k_sources, int max_m, int batch, int max_chunks);
 // place them: `ws_area` is the device address of that area, `tmap_host`/`tmap_dev` one 128-byte descriptor slot
-void tc_setup_absorb(TcState &tc, const kvcar_config &cfg, int max_k_sources, int max_m, int batch, char *ws_area,
-                     char *tmap_host, char *tmap_dev);
+void tc_setup_absorb(TcState &tc, const kvcar_config &cfg, int max_k_sources, int max_m, int batch, int max_chunks,
+                     char *ws_area, char *tmap_host, char *tmap_dev);
+// the merge of the tiles after a launch that took the absorbed V form (tc.last_mode == 2)
+cudaError_t tc_launch_combine_absorbed(const TcState &tc, const DecodeArgs &a, const SeqList &seqs, cudaStream_t st);
 
 // Build the TMA descriptors and the per-layer job tables into the host image of the
 // weights buffer (at tmap_off / part_off) and decide per layer whether the tensor-core

@@ -29,6 +29,7 @@ def main(argv=None) -> int:
     ap.add_argument("--cluster", type=int, default=0)
     ap.add_argument("--jobs", type=int, default=14, help="jobs to list")
     ap.add_argument("--absorbed", action="store_true", help="pass KVCAR_ABSORBED")
+    ap.add_argument("--absorbed-v", action="store_true", help="with --absorbed: KVCAR_ABSORBED_V as well")
     ap.add_argument("--json", default=None, help="also write the raw stamps here")
     args = ap.parse_args(argv)
 
@@ -71,7 +72,8 @@ def main(argv=None) -> int:
     for _ in range(3):
         e0.record()
         sess.ctx.decode_attention(args.layer, seqs, q.data_ptr(), out.data_ptr(),
-                                  B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if args.absorbed else 0), sess.stream())
+                                  B.INCLUDE_CURRENT_EXACT | (B.ABSORBED if args.absorbed else 0) |
+                                  (B.ABSORBED_V if args.absorbed and args.absorbed_v else 0), sess.stream())
         e1.record()
         torch.cuda.synchronize()
     sess.ctx.sync_status(sess.stream())
@@ -96,8 +98,8 @@ def report(ev, n_list):
     t_zero = min(iss[0][0], ep[0][0])
     jobs, cur, last = [], None, None
     for t, tag in iss:
-        if tag in (0x11, 0x12, 0x13):
-            cur = dict(kind=tag & 3, t0=t, wait=0, issue=0, slabs=0, prev=t)
+        if tag in (0x11, 0x12, 0x13, 0x14):
+            cur = dict(kind=tag & 7, t0=t, wait=0, issue=0, slabs=0, prev=t)
             jobs.append(cur)
         elif tag == 0x30:
             cur["wait"] += t - cur["prev"]
@@ -118,7 +120,7 @@ def report(ev, n_list):
             c["seen"] = t
         elif ph == 3:
             c["done"] = t
-    names = {1: "hidden chunk", 2: "head group", 3: "K scores"}
+    names = {1: "hidden chunk", 2: "head group", 3: "K scores", 4: "V sums"}
     print("job  kind          start     cycles slabs   wait  issue | epilogue: job seen complete  work")
     for i, (j, e) in enumerate(zip(jobs, ejobs)):
         if i >= n_list or "t1" not in j or "done" not in e:
@@ -129,7 +131,7 @@ def report(ev, n_list):
     span = iss[-1][0] - iss[0][0]
     print(f"issuer: {len(done)} jobs, {sum(j['slabs'] for j in done)} slabs in {span} cycles; waiting {sum(j['wait'] for j in done)},"
           f" issuing {sum(j['issue'] for j in done)}, between jobs {sum(done[i + 1]['t0'] - done[i]['t1'] for i in range(len(done) - 1))}")
-    for kind in (1, 2, 3):
+    for kind in (1, 2, 3, 4):
         sel = [j for j in done if j["kind"] == kind]
         if sel:
             print(f"  {names[kind]} jobs: {len(sel)}, mean {sum(j['t1'] - j['t0'] for j in sel) / len(sel):.0f} cycles,"

@@ -115,7 +115,8 @@ class Pair:
         """Returns (gpu [n,Hq,hd] float64, oracle rows or None, row indices the oracle covers)."""
         dq = self.s.to_device(q)
         out = torch.empty_like(dq)
-        flags = (B.INCLUDE_CURRENT_EXACT if include_current else 0) | (B.ABSORBED if absorbed else 0)
+        flags = (B.INCLUDE_CURRENT_EXACT if include_current else 0) | \
+                (B.ABSORBED if absorbed else 0) | (B.ABSORBED_V if absorbed == "kv" else 0)
         self.s.ctx.decode_attention(layer, list(seqs), dq.data_ptr(), out.data_ptr(), flags, self.s.stream())
         self.s.ctx.sync_status(self.s.stream())
         got = out.float().cpu().numpy().astype(np.float64)
@@ -131,7 +132,8 @@ class Pair:
         """append + attention of one layer through the single-call entry point; same return as attention()."""
         dk, dv, dq = self.s.to_device(k), self.s.to_device(v), self.s.to_device(q)
         out = torch.empty_like(dq)
-        flags = (B.INCLUDE_CURRENT_EXACT if include_current else 0) | (B.ABSORBED if absorbed else 0)
+        flags = (B.INCLUDE_CURRENT_EXACT if include_current else 0) | \
+                (B.ABSORBED if absorbed else 0) | (B.ABSORBED_V if absorbed == "kv" else 0)
         self.s.ctx.step_layer(layer, list(seqs), dk.data_ptr(), dv.data_ptr(), dq.data_ptr(), out.data_ptr(), flags,
                               self.s.stream())
         self.s.ctx.sync_status(self.s.stream())

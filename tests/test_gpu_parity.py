@@ -378,6 +378,35 @@ def test_int8_latent_rows_match_the_oracle(cfg):
     assert comp < 0.55 * plain.s.ctx.cache_bytes_per_token()[0]
 
 
+@pytest.mark.parametrize("shape", ["gpt2", "group2_narrow"])
+def test_absorbed_last_layer_on_both_sides_matches_the_oracle(shape):
+    """KVCAR_ABSORBED | KVCAR_ABSORBED_V: the V side too - a tile hands on sum_t p_t a_t (m values per query head) and
+    W4_h is applied once per sequence and head when the tiles are merged; no restored K or V row is ever formed.
+    Same tolerance as the plain form; ragged lengths, reuse (several V sources per layer), two steps, and the
+    output must also agree with the plain form of the same context."""
+    if shape == "gpt2":            # 12 heads, hidden 576: nine slabs, the last feature chunk repeats a slab
+        w = synth.scaled(synth.CONFIGS["c2"], n_layers=3, batch=5, cached_tokens=0, decode_steps=2, reuse_frac=0.25)
+    else:                          # 8 query / 4 KV heads, hidden 192: three slabs
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, n_q_heads=8, n_kv_heads=4, latent_full=128, batch=5,
+                         cached_tokens=0, decode_steps=2, reuse_frac=0.25)
+    pps = 34
+    p = Pair(w, max_seqs=5, max_pages=5 * pps, max_pages_per_seq=pps, kernel=B.KERNEL_TENSOR)
+    seqs = [0, 1, 2, 3, 4]
+    p.open(seqs)
+    for s_, n in zip(seqs, (2100, 2049, 2111, 2050, 2064)):     # 17 tiles each: 85 tiles, 43 pairs
+        p.prefill([s_], n)
+    for step in range(2):
+        res = p.decode_step(seqs, step, absorbed="kv")
+        _check_step(res, "bf16", f"absorbed K and V {shape} step {step}")
+    # against the plain form on the same cache (one more layer call each way, no append)
+    q = np.stack([synth.make_q(w, 1, s_, 7) for s_ in seqs])
+    got_a, _, _ = p.attention(1, seqs, q, absorbed="kv")
+    got_p, ref, rows = p.attention(1, seqs, q)
+    assert_close(got_a[rows], ref, "bf16", "absorbed K and V, layer 1")
+    assert np.max(np.abs(got_a - got_p)) < 2e-2
+    assert np.max(np.abs(got_a - got_p)) > 0.0   # the other form did run
+
+
 @pytest.mark.parametrize("shape", ["gpt2", "tinyllama", "group2_narrow"])
 def test_absorbed_last_layer_matches_the_oracle(shape):
     """KVCAR_ABSORBED: a head's scores are taken as a.(W4_h^T q) + q.b4_h from the activated hidden vectors, the
