@@ -37,7 +37,7 @@ def _reused_heads(w):
     return {(l, h) for l in range(w.n_layers) for h in range(w.n_kv_heads) if src[l * w.n_kv_heads + h] >= 0}
 
 
-def _run(w, sampled, steps=1, fused=False, compress=True):
+def _run(w, sampled, steps=1, fused=False, compress=True, absorbed=False):
     pps = (w.cached_tokens + steps + w.page_tokens - 1) // w.page_tokens
     p = Pair(w, max_seqs=w.batch, max_pages=w.batch * pps, max_pages_per_seq=pps, kernel=B.KERNEL_AUTO,
              compress=compress)
@@ -50,7 +50,7 @@ def _run(w, sampled, steps=1, fused=False, compress=True):
     worst = 0.0
     pairs = set()
     for step in range(steps):
-        res = p.decode_step(seqs, step, fused=fused)
+        res = p.decode_step(seqs, step, fused=fused, absorbed=absorbed)
         for l, (got, ref, rows) in res.items():
             assert rows == sorted(sampled)
             err, _ = assert_close(got[rows], ref, w.storage, f"{w.name} step {step} layer {l}")
@@ -97,6 +97,16 @@ def test_config5_batch_sweep_point_sampled():
     w = synth.with_batch(synth.CONFIGS["c5"], 32)
     _, _, _, pairs, hit = _run(w, [0, 5, 11, 17, 23, 31], steps=2)
     assert len(pairs) == 72 and hit == _reused_heads(w)
+
+
+@pytest.mark.parametrize("form", [True, "kv"], ids=["k", "k_and_v"])
+def test_config5_absorbed_forms_sampled(form):
+    """The same point of the batch sweep (GPT-2 shape, 4096 cached tokens, batch 32, all 12 layers with their reuse
+    sources) through the absorbed last decoder layer - K side only, and both sides: two steps through the single-call
+    step, sequences 0, 9, 16 and 31 against the oracle (48 (sequence, layer) pairs, every reused head)."""
+    w = synth.with_batch(synth.CONFIGS["c5"], 32)
+    _, _, _, pairs, hit = _run(w, [0, 9, 16, 31], steps=2, fused=True, absorbed=form)
+    assert len(pairs) == 48 and hit == _reused_heads(w)
 
 
 def test_config5_largest_batch_single_call_step_sampled():
