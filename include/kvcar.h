@@ -220,8 +220,9 @@ kvcar_status kvcar_advance(kvcar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, 
  * same for V, sum_t p_t v'_t = W4_h (sum_t p_t a_t) + b4_h sum_t p_t: a tile
  * hands on sum_t p_t a_t (m values per query head) and the last layer is applied
  * once per sequence and head when the tiles are merged; the probabilities enter
- * that product rounded to the storage type.  For at most 16 query heads; ignored
- * elsewhere.
+ * that product rounded to the storage type.  For at most 32 query heads and
+ * hidden layers whose feature chunks fit one accumulator buffer (576 columns with
+ * up to 16 query heads, 512 with up to 32); ignored elsewhere.
  */
 kvcar_status kvcar_decode_attention(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                     const void *q, void *out, uint32_t flags, void *stream);

@@ -1143,15 +1143,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             const int sa = min(2 * c, ks2 - 2);
                             const int f = sa * 64 + row;
                             const bool repeated = 2 * c > ks2 - 2 && row < 64;  // slab already covered by the chunk before
-                            float u[16];
                             const uint32_t ta = acc + (uint32_t)(c * 2 * lay.nq_pad + lay.nq_pad * (int)rank);
-                            tmem_ld8(ta, u);
-                            tmem_ld8(ta + 8u, u + 8);
-                            tmem_ld_wait();
-                            if (!repeated && f < m) {
+                            for (int q0 = 0; q0 < lay.nq_pad; q0 += 16) {
+                                float u[16];
+                                tmem_ld8(ta + (uint32_t)q0, u);
+                                tmem_ld8(ta + (uint32_t)q0 + 8u, u + 8);
+                                tmem_ld_wait();
+                                if (!repeated && f < m) {
 #pragma unroll
-                                for (int ql = 0; ql < 16; ++ql)
-                                    if ((mask >> ql) & 1u) ub[(int64_t)ql * lay.m_pad_u + f] = u[ql];
+                                    for (int ql = 0; ql < 16; ++ql)
+                                        if ((mask >> (q0 + ql)) & 1u) ub[(int64_t)(q0 + ql) * lay.m_pad_u + f] = u[ql];
+                                }
                             }
                         }
                     }
@@ -1299,6 +1301,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 inline uint32_t up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
 PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslots, int nslot, bool pop = false) {
+    const int nq_pad_pop = nq_local <= 16 ? 16 : 32;
     PairLaunch l{};
     const int ks_hid = (max_m + 63) / 64;
     uint32_t o = 0;
@@ -1319,10 +1322,10 @@ PairLaunch make_launch(int nq_local, int group, int max_m, int max_in, int pslot
     if (l.group_mma) o = up(o + (uint32_t)nq_local * QBS * 2, 16);
     l.off_pb = o;
     if (l.group_mma) o = up(o + 2u * (uint32_t)nq_local * PBS * 2, 16);
-    if (pop) {  // absorbed V: the tile's probabilities as a column operand, 16 rows x 256 B, on a swizzle boundary
+    if (pop) {  // absorbed V: the tile's probabilities as a column operand, 16 or 32 rows x 256 B, on a swizzle boundary
         o = up(o, 1024);
         l.off_pop = o;
-        o += 16 * 256;
+        o += (uint32_t)nq_pad_pop * 256;
     }
     l.off_bar = o;
     l.nslot = nslot;
@@ -1393,10 +1396,10 @@ bool build_part(const LayerPlan &lp, const TcSrc (*srcs)[MAX_SRC], int h_lo, int
                 n = 0;  // no head groups
             }
             if (absorbed_v && which == 1) {
-                // one job for the whole source: at most 16 query heads, at least two hidden slabs (the row operand
-                // spans two), and all 128-feature chunks side by side in one 256-column accumulator buffer
-                const int ks2 = (sp.m + 63) / 64;
-                if (nj == TC_MAX_JOBS || (h_hi - h_lo) * group > 16 || ks2 < 2 || ((ks2 + 1) / 2) * 32 > 256) return false;
+                // one job for the whole source: at least two hidden slabs (the row operand spans two), and all
+                // 128-feature chunks side by side in one 256-column accumulator buffer (2 x 16 or 2 x 32 columns each)
+                const int ks2 = (sp.m + 63) / 64, nq = (h_hi - h_lo) * group, cols = 2 * (nq <= 16 ? 16 : 32);
+                if (nj == TC_MAX_JOBS || nq > TC_ABS_MAX_Q || ks2 < 2 || ((ks2 + 1) / 2) * cols > 256) return false;
                 TcJob &jb = out.jobs[which][nj++];
                 jb.kind = 4;
                 jb.src = (uint8_t)ns;
@@ -1614,7 +1617,7 @@ cudaError_t tc_launch_combine_absorbed(const TcState &tc, const DecodeArgs &a, c
 // absorbed V side: bytes of the U vectors (0 where the form is not taken: more than 16 query heads, or more than
 // 512 tiles per sequence, which the merge kernel's weight table does not hold)
 static size_t absorb_u_bytes(const kvcar_config &cfg, int max_m, int batch, int max_chunks) {
-    if (cfg.n_q_heads > 16 || max_chunks > 512) return 0;
+    if (cfg.n_q_heads > TC_ABS_MAX_Q || max_chunks > 512) return 0;
     const size_t m_pad = ((size_t)max_m + 63) / 64 * 64;
     return (size_t)batch * max_chunks * cfg.n_q_heads * m_pad * sizeof(float);
 }
@@ -1740,7 +1743,7 @@ void tc_setup(TcState &tc, const kvcar_config &cfg, const LayerPlan *plans, int 
         }
         if (!lc.split_ok[0]) continue;
         lc.abs_ok = cfg.n_q_heads <= TC_ABS_MAX_Q && build_part(plans[l], srcs, 0, cfg.n_kv_heads, parts[7], true, group) ? 1 : 0;
-        lc.absv_ok = lc.abs_ok && cfg.n_q_heads <= 16 &&
+        lc.absv_ok = lc.abs_ok &&
                      pick_nslot(cfg.n_kv_heads * group, group, max_m, max_in, pslots, true) >= 3 &&
                      build_part(plans[l], srcs, 0, cfg.n_kv_heads, parts[8], true, group, true) ? 1 : 0;
         lc.ok = 1;

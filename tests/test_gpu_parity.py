@@ -378,7 +378,7 @@ def test_int8_latent_rows_match_the_oracle(cfg):
     assert comp < 0.55 * plain.s.ctx.cache_bytes_per_token()[0]
 
 
-@pytest.mark.parametrize("shape", ["gpt2", "group2_narrow"])
+@pytest.mark.parametrize("shape", ["gpt2", "group2_narrow", "tinyllama"])
 def test_absorbed_last_layer_on_both_sides_matches_the_oracle(shape):
     """KVCAR_ABSORBED | KVCAR_ABSORBED_V: the V side too - a tile hands on sum_t p_t a_t (m values per query head) and
     W4_h is applied once per sequence and head when the tiles are merged; no restored K or V row is ever formed.
@@ -386,6 +386,8 @@ def test_absorbed_last_layer_on_both_sides_matches_the_oracle(shape):
     output must also agree with the plain form of the same context."""
     if shape == "gpt2":            # 12 heads, hidden 576: nine slabs, the last feature chunk repeats a slab
         w = synth.scaled(synth.CONFIGS["c2"], n_layers=3, batch=5, cached_tokens=0, decode_steps=2, reuse_frac=0.25)
+    elif shape == "tinyllama":     # 32 query / 4 KV heads (two 32-column blocks per chunk), hidden 192
+        w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, batch=5, cached_tokens=0, decode_steps=2, reuse_frac=0.25)
     else:                          # 8 query / 4 KV heads, hidden 192: three slabs
         w = synth.scaled(synth.CONFIGS["c3"], n_layers=3, n_q_heads=8, n_kv_heads=4, latent_full=128, batch=5,
                          cached_tokens=0, decode_steps=2, reuse_frac=0.25)
