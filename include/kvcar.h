@@ -46,7 +46,8 @@ typedef enum {
     KVCAR_ERR_WORKSPACE = 4,     /* bound buffers too small for the request          */
     KVCAR_ERR_UNSUPPORTED = 5,   /* shape outside what the kernels handle            */
     KVCAR_ERR_CUDA = 6,          /* a CUDA runtime/driver call failed                */
-    KVCAR_ERR_DEVICE_TIMEOUT = 7 /* a bounded device-side wait ran out               */
+    KVCAR_ERR_DEVICE_TIMEOUT = 7,/* a bounded device-side wait ran out               */
+    KVCAR_ERR_GUARD = 8          /* kvcar_debug_check found memory it guards altered */
 } kvcar_status;
 
 typedef enum { KVCAR_F32 = 0, KVCAR_BF16 = 1 } kvcar_dtype;
@@ -342,6 +343,18 @@ const char *kvcar_last_error(kvcar_ctx *ctx);
  * wait of the fused kernel ends this way when it runs out (their limit is 2 s);
  * nothing traps and the context stays usable. */
 kvcar_status kvcar_debug_expire_wait(kvcar_ctx *ctx, uint64_t limit_ns, void *stream);
+/* Stand-in for a memory checker, callable at any point between steps.  The pool
+ * buffer carries 256 guard bytes behind each of its regions (every layer's K and V
+ * pool, their int8 row parameters, the per-layer current-token rows), filled with
+ * a fixed byte by kvcar_bind_memory; no kernel has a reason to write them.  The
+ * call brings the device tables up to date, waits for `stream`, reads the guards
+ * and the device copies of the page table and sequence lengths back and compares
+ * them with the fill byte and with the allocator's host-side tables.  Returns
+ * KVCAR_OK, or KVCAR_ERR_GUARD with *what = 1 (guard byte altered; *where = byte
+ * offset in the pool buffer), 2 (page-table entry; *where = sequence *
+ * max_pages_per_seq + index) or 3 (sequence length; *where = sequence).  Host
+ * pointers; synchronises the stream; not for the timed path. */
+kvcar_status kvcar_debug_check(kvcar_ctx *ctx, void *stream, int32_t *what, int64_t *where);
 
 /* ---- choosing the reuse map (Alg. 2, its first three steps) -------------------
  *

@@ -23,7 +23,7 @@ ABSORBED_V = 4
 MAX_BATCH = 512
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "STATE", 3: "OOM_PAGES", 4: "WORKSPACE", 5: "UNSUPPORTED",
-                6: "CUDA", 7: "DEVICE_TIMEOUT"}
+                6: "CUDA", 7: "DEVICE_TIMEOUT", 8: "GUARD"}
 
 EXPORTS = [
     "kvcar_create", "kvcar_destroy", "kvcar_set_reuse_map", "kvcar_set_autoencoder", "kvcar_required_bytes",
@@ -32,7 +32,7 @@ EXPORTS = [
     "kvcar_step_layer", "kvcar_step_layer_host",
     "kvcar_debug_resolve", "kvcar_debug_locate", "kvcar_seq_len", "kvcar_pool_layout", "kvcar_pool_quant_layout",
     "kvcar_cache_bytes_per_token", "kvcar_layer_work_per_token", "kvcar_layer_work_absorbed", "kvcar_launch_count", "kvcar_layer_kernel", "kvcar_sync_status",
-    "kvcar_last_error", "kvcar_debug_expire_wait",
+    "kvcar_last_error", "kvcar_debug_expire_wait", "kvcar_debug_check",
     "kvcar_head_l1_scratch_bytes", "kvcar_head_l1_distance", "kvcar_reuse_map_from_l1",
 ]
 
@@ -114,6 +114,7 @@ def _load(trace: bool = False) -> C.CDLL:
         "kvcar_layer_kernel": [vp, i32, ip],
         "kvcar_sync_status": [vp, vp],
         "kvcar_debug_expire_wait": [vp, C.c_uint64, vp],
+        "kvcar_debug_check": [vp, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int64)],
         "kvcar_head_l1_scratch_bytes": [i32, i32, C.c_int64, C.POINTER(sz)],
         "kvcar_head_l1_distance": [i32, i32, i32, i32, vp, C.c_int64, vp, sz, vp, vp],
         "kvcar_reuse_map_from_l1": [C.POINTER(C.c_float), i32, i32, i32, ip],
@@ -337,3 +338,9 @@ class Context:
 
     def debug_expire_wait(self, limit_ns: int, stream: int = 0):
         self._check(self.lib.kvcar_debug_expire_wait(self._h, limit_ns, stream))
+
+    def debug_check(self, stream: int = 0):
+        """(status, what, where) of kvcar_debug_check; status 0 = guards and device tables intact."""
+        what, where = C.c_int32(), C.c_int64()
+        st = self.lib.kvcar_debug_check(self._h, stream, C.byref(what), C.byref(where))
+        return st, what.value, where.value

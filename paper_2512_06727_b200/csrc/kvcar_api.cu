@@ -8,6 +8,8 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "kvcar_internal.h"
 #include "kvcar_tc.h"
 
@@ -27,6 +29,16 @@ struct Resolved {
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// A named range around each call that enqueues work, for timeline tools that read NVTX; without such a tool
+// attached the two calls return at once.
+struct Range {
+    explicit Range(const char *name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
+
+constexpr size_t GUARD_BYTES = 256;        // behind every region of the pool buffer; no kernel writes there
+constexpr unsigned char GUARD_FILL = 0xA5;
 
 }  // namespace
 
@@ -48,6 +60,7 @@ struct kvcar_ctx {
     std::vector<char> open;
     std::vector<int4> pending;  // device table updates not yet enqueued
     bool table_dirty_all = false;
+    std::vector<size_t> guard_off;  // offsets (pool buffer) of the GUARD_BYTES-byte guard regions, filled at bind
 
     // device buffers and layout
     char *pool = nullptr, *weights = nullptr, *ws = nullptr;
@@ -118,6 +131,7 @@ void compute_layout(kvcar_ctx *c) {
     c->qparam_off.assign(nl * 2, 0);
     c->quant.assign(nl * 2, 0);
     size_t off = 0;
+    c->guard_off.clear();
     c->max_d = c->max_m = c->max_in = 0;
     for (int i = 0; i < nl * 2; ++i) {
         c->width[i] = stored_width(c, i / 2, i % 2);
@@ -126,11 +140,15 @@ void compute_layout(kvcar_ctx *c) {
         if (g.latent_quant && a.set) {  // Eq. 4: one byte per element, then (scale, zero-point) per row
             c->quant[i] = 1;
             off = align_up(off + rows * c->width[i], 256);
+            c->guard_off.push_back(off);
+            off += GUARD_BYTES;
             c->qparam_off[i] = off;
             off = align_up(off + rows * 2 * sizeof(float), 256);
         } else {
             off = align_up(off + rows * c->width[i] * c->elem, 256);
         }
+        c->guard_off.push_back(off);  // 256 guard bytes behind every pool region
+        off += GUARD_BYTES;
         if (a.set) {
             c->max_d = std::max(c->max_d, a.latent);
             c->max_m = std::max(c->max_m, a.hidden);
@@ -142,6 +160,8 @@ void compute_layout(kvcar_ctx *c) {
     for (int i = 0; i < nl * 2; ++i) {
         c->cur_off[i] = off;
         off = align_up(off + (size_t)g.max_seqs * W * c->elem, 256);
+        c->guard_off.push_back(off);
+        off += GUARD_BYTES;
     }
     c->pool_bytes = off;
 
@@ -419,6 +439,7 @@ kvcar_status kvcar_required_bytes(kvcar_ctx *c, size_t *pool, size_t *weights, s
 
 kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void *weights, size_t weights_bytes,
                                void *workspace, size_t workspace_bytes, void *stream) {
+    Range range_("kvcar_bind_memory");
     if (!c || !pool || !weights || !workspace) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
     if (c->bound) return fail(c, KVCAR_ERR_STATE, "memory already bound");
     if (((uintptr_t)pool | (uintptr_t)weights | (uintptr_t)workspace) & 255)
@@ -613,6 +634,9 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
         if (static_scratch_for_current_device(&p) != cudaSuccess) cudaGetLastError();
         c->static_scratch = p;
     }
+    for (size_t off : c->guard_off)
+        if (cudaMemsetAsync(c->pool + off, GUARD_FILL, GUARD_BYTES, st) != cudaSuccess)
+            return cuda_fail(c, cudaGetLastError(), "guard fill");
     c->bound = true;
     c->pending.clear();
     // re-queue what host bookkeeping already holds (sequences opened / pages reserved before binding)
@@ -662,6 +686,7 @@ static kvcar_status enqueue_encode(kvcar_ctx *c, int32_t layer, const int32_t *s
 
 kvcar_status kvcar_encode_append(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens,
                                  const void *k, const void *v, void *stream) {
+    Range range_("kvcar_encode_append");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
     if (layer < 0 || layer >= c->cfg.n_layers || !k || !v || n_tokens <= 0)
@@ -712,6 +737,7 @@ static kvcar_status enqueue_encode(kvcar_ctx *c, int32_t layer, const int32_t *s
 
 kvcar_status kvcar_encode_append_tensor(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                         int32_t n_tokens, const void *k, const void *v, void *stream) {
+    Range range_("kvcar_encode_append_tensor");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
     if (layer < 0 || layer >= c->cfg.n_layers || !k || !v || n_tokens <= 0)
@@ -757,6 +783,7 @@ kvcar_status kvcar_encode_append_tensor(kvcar_ctx *c, int32_t layer, const int32
 }
 
 kvcar_status kvcar_advance(kvcar_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t n_tokens, void *stream) {
+    Range range_("kvcar_advance");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     if (!check_seqs(c, seqs, n_seqs) || n_tokens <= 0) return fail(c, KVCAR_ERR_INVALID_ARG, "bad sequence list");
     const int P = c->cfg.page_tokens;
@@ -852,6 +879,7 @@ static kvcar_status check_decode_args(kvcar_ctx *c, int32_t layer, const int32_t
 
 kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *q,
                                     void *out, uint32_t flags, void *stream) {
+    Range range_("kvcar_decode_attention");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     kvcar_status s = check_decode_args(c, layer, seqs, n_seqs, q, out, flags);
     if (s != KVCAR_OK) return s;
@@ -868,6 +896,7 @@ kvcar_status kvcar_decode_attention(kvcar_ctx *c, int32_t layer, const int32_t *
 
 kvcar_status kvcar_step_layer(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs, const void *k,
                               const void *v, const void *q, void *out, uint32_t flags, void *stream) {
+    Range range_("kvcar_step_layer");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     kvcar_status s = check_decode_args(c, layer, seqs, n_seqs, q, out, flags);
     if (s != KVCAR_OK) return s;
@@ -914,6 +943,7 @@ kvcar_status kvcar_step_layer(kvcar_ctx *c, int32_t layer, const int32_t *seqs, 
 kvcar_status kvcar_step_layer_host(kvcar_ctx *c, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                    const void *k_host, const void *v_host, const void *q_host, void *out_host,
                                    uint32_t flags, void *stream) {
+    Range range_("kvcar_step_layer_host");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
     if (!k_host || !v_host || !q_host || !out_host) return fail(c, KVCAR_ERR_INVALID_ARG, "null host buffer");
@@ -1097,6 +1127,48 @@ kvcar_status kvcar_debug_expire_wait(kvcar_ctx *c, uint64_t limit_ns, void *stre
     return KVCAR_OK;
 }
 
+kvcar_status kvcar_debug_check(kvcar_ctx *c, void *stream, int32_t *what, int64_t *where) {
+    if (!c || !what || !where) return fail(c, KVCAR_ERR_INVALID_ARG, "null argument");
+    if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
+    *what = 0;
+    *where = -1;
+    cudaStream_t st = (cudaStream_t)stream;
+    kvcar_status fs = flush_tables(c, st);
+    if (fs != KVCAR_OK) return fs;
+    const kvcar_config &g = c->cfg;
+    const int mp = g.max_pages_per_seq;
+    std::vector<unsigned char> guards(c->guard_off.size() * GUARD_BYTES);
+    std::vector<int32_t> bt((size_t)g.max_seqs * mp), ln(g.max_seqs);
+    cudaError_t e = cudaSuccess;
+    for (size_t i = 0; i < c->guard_off.size() && e == cudaSuccess; ++i)
+        e = cudaMemcpyAsync(&guards[i * GUARD_BYTES], c->pool + c->guard_off[i], GUARD_BYTES, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(bt.data(), c->ws + c->bt_off, bt.size() * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ln.data(), c->ws + c->len_off, ln.size() * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "read-back for the check");
+    for (size_t i = 0; i < guards.size(); ++i)
+        if (guards[i] != GUARD_FILL) {
+            *what = 1;
+            *where = (int64_t)(c->guard_off[i / GUARD_BYTES] + i % GUARD_BYTES);
+            return fail(c, KVCAR_ERR_GUARD, "a guard region of the pool buffer was written");
+        }
+    for (int s = 0; s < g.max_seqs; ++s) {
+        if (!c->open[s]) continue;
+        for (size_t i = 0; i < c->table[s].size(); ++i)
+            if (bt[(size_t)s * mp + i] != c->table[s][i]) {
+                *what = 2;
+                *where = (int64_t)s * mp + (int64_t)i;
+                return fail(c, KVCAR_ERR_GUARD, "the device page table differs from the allocator's");
+            }
+        if (ln[s] != c->len[s]) {
+            *what = 3;
+            *where = s;
+            return fail(c, KVCAR_ERR_GUARD, "a device sequence length differs from the host's");
+        }
+    }
+    return KVCAR_OK;
+}
+
 }  // extern "C"
 
 // =============================================================================
@@ -1133,6 +1205,7 @@ cudaError_t static_scratch_for_current_device(float **out) {
 extern "C" kvcar_status kvcar_decode_attention_static(kvcar_ctx *c, int32_t layer, const int32_t *seqs,
                                                       int32_t n_seqs, const void *q, void *out, uint32_t flags,
                                                       void *stream) {
+    Range range_("kvcar_decode_attention_static");
     if (!c) return KVCAR_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, KVCAR_ERR_STATE, "bind memory first");
     if (layer < 0 || layer >= c->cfg.n_layers || !q || !out)

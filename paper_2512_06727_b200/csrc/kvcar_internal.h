@@ -124,7 +124,7 @@ size_t decode_generic_smem(int hq, int hd, int max_d, int max_m);
 // Bulk encoder + append on the tensor cores (kvcar_prefill_tc.cu): bf16 storage, both K and V of the layer with an
 // autoencoder, head_dim 64, hidden and latent widths multiples of 16.  Rows are worked through in blocks of
 // PREFILL_TC_ROWS; `hid` is a bf16 scratch of prefill_tc_scratch_bytes(max hidden width) bytes.
-constexpr int PREFILL_TC_ROWS = 8192;
+constexpr int PREFILL_TC_ROWS = 32768;
 struct PrefillTcArgs {
     const EncPlan *plan_dev;    // this layer's [K, V] plans on the device
     const EncPlan *plan_host;   // the same two plans, host copy (widths and weight pointers for the tensor maps)

@@ -355,6 +355,36 @@ def test_device_side_wait_that_runs_out_is_reported_and_the_context_stays_usable
     _check_step(p.decode_step([0, 1], 0), "bf16", "after a timed-out wait")
 
 
+@pytest.mark.parametrize("cfg,quant", [("c2", False), ("c3", False), ("c2", True)])
+def test_guard_regions_and_device_tables_survive_prefill_and_decode(cfg, quant):
+    """Stand-in for a memory checker: 256 guard bytes behind every pool region (K and V pools, int8 row parameters,
+    current-token rows) keep their fill through bulk and per-token encoding, decode steps on full and ragged
+    pages, and a sequence that fills its last reserved page to the end; the device page table and lengths equal the
+    allocator's.  A byte planted by the test just behind layer 0's K pool is then found and located."""
+    w = synth.scaled(synth.CONFIGS[cfg], n_layers=3, batch=3, reuse_frac=0.25)
+    p = Pair(w, max_seqs=3, max_pages=9, max_pages_per_seq=3, latent_quant=quant)
+    p.open([0, 1, 2])
+    p.prefill([0], 3 * 64 - 1)          # one step short of the end of its last page
+    p.prefill([1], 65)
+    p.prefill([2], 1)
+    assert p.s.ctx.debug_check(p.s.stream()) == (0, 0, -1)
+    p.decode_step([0, 1, 2], 0)         # sequence 0 now ends exactly at the end of the pool rows reserved for it
+    assert p.s.ctx.debug_check(p.s.stream()) == (0, 0, -1)
+    off, pitch, width = p.s.ctx.pool_layout(0, 0)
+    rows = p.s.ctx.cfg.max_pages * p.s.ctx.cfg.page_tokens
+    guard = (off + rows * pitch + 255) // 256 * 256
+    base = p.s._aligned(p.s.pool) - p.s.pool.data_ptr()
+    torch.cuda.synchronize()
+    assert int(p.s.pool[base + guard + 7]) == 0xA5
+    p.s.pool[base + guard + 7] = 0
+    torch.cuda.synchronize()
+    st, what, where = p.s.ctx.debug_check(p.s.stream())
+    assert (st, what, where) == (8, 1, guard + 7)
+    p.s.pool[base + guard + 7] = 0xA5
+    torch.cuda.synchronize()
+    assert p.s.ctx.debug_check(p.s.stream()) == (0, 0, -1)
+
+
 @pytest.mark.parametrize("cfg", ["c2", "c3"])
 def test_int8_latent_rows_match_the_oracle(cfg):
     """Sec. "Quantization" on top of the autoencoders (Table 5's combination): every cached latent row is stored
