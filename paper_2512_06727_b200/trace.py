@@ -90,6 +90,44 @@ def main(argv=None) -> int:
     return 0
 
 
+def ring_legs(ev):
+    """The staging ring's round trip in the head-group phase, from the producers' and the issuer's stamps of the
+    leader CTA: both producers stamp every slab once they are past its place (the one that loads it after the load
+    is issued), the issuer stamps operands seen (0x30) and products + release issued (0x31).  Slab i of a head-group
+    job re-uses the place of slab i - 3 (a ring of three places, as at the GPT-2 shape)."""
+    iss = ev["0.2"]
+    prod = [[t for t, g in ev[f"0.{r}"] if g in (2, 3)] for r in (0, 1)]
+    seen, rel, kind = [], [], []
+    k = None
+    for t, tag in iss:
+        if tag in (0x11, 0x12, 0x13, 0x14):
+            k = tag & 7
+        elif tag == 0x30:
+            seen.append(t)
+            kind.append(k)
+        elif tag == 0x31:
+            rel.append(t)
+    n = min(len(seen), len(rel), len(prod[0]), len(prod[1]))
+    if n < 8:
+        return
+    load, free, gap = [], [], []
+    for i in range(n):
+        if kind[i] != 2:
+            continue
+        issued = max(prod[0][i], prod[1][i])
+        load.append(seen[i] - issued)
+        if i + 3 < n and kind[i + 3] == 2:
+            free.append(min(prod[0][i + 3], prod[1][i + 3]) - rel[i])
+        if i > 0 and kind[i - 1] == 2:
+            gap.append(seen[i] - rel[i - 1])
+    if not load or not free:
+        return
+    med = lambda v: sorted(v)[len(v) // 2]
+    print(f"  head-group ring: load issued -> operands seen by the issuer: median {med(load)} cycles; products + release issued"
+          f" (slab i) -> place seen free for slab i+3: median {med(free)}; release issued -> next operands seen: median"
+          f" {med(gap)}; issue of a slab (0x30 -> 0x31): median {med([r - s for r, s, k in zip(rel, seen, kind) if k == 2])}")
+
+
 def report(ev, n_list):
     iss, ep = ev["0.2"], ev["0.3"]
     if not iss or not ep:
@@ -136,6 +174,7 @@ def report(ev, n_list):
         if sel:
             print(f"  {names[kind]} jobs: {len(sel)}, mean {sum(j['t1'] - j['t0'] for j in sel) / len(sel):.0f} cycles,"
                   f" {sum(j['t1'] - j['t0'] for j in sel) / max(1, sum(j['slabs'] for j in sel)):.0f} per slab")
+    ring_legs(ev)
     for kind, nm in ((4, "hidden chunk"), (5, "K head group"), (6, "V head group")):
         sel = [e for e in ejobs if e["kind"] == kind and "done" in e and "seen" in e]
         if sel:
