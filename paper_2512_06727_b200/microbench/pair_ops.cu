@@ -4,8 +4,9 @@
 // (3) shared-memory bytes per clock that 1, 2 or 4 threads of an SM get from tensor loads of L2-resident data;
 // (4) what a completed mbarrier.try_wait, an expect-tx, a tensor load and a mapa cost their thread on an idle SM, and
 // how long a 16-KB load takes to land; (5) the rate of tensor loads into shared memory while the pair's tensor pipe
-// runs products out of the same shared memory, and the products' rate meanwhile.  Every wait is bounded; results go
-// to stdout.
+// runs products out of the same shared memory, and the products' rate meanwhile; (6) the issuer's and a producer's loop
+// while eight other warps of the CTA sleep, compute, use shared memory or read tensor memory.  Every wait is bounded;
+// results go to stdout.
 //   nvcc -gencode arch=compute_100a,code=sm_100a -O3 -std=c++17 -I ../csrc -o pair_ops pair_ops.cu -lcuda && ./pair_ops
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -315,6 +316,147 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1) mix_kernel(c
     }
 }
 
+
+// test 6: the issuer's and a producer's loop while eight other warps of each CTA do one kind of work.  Issuer: per
+// round one try_wait, one fence, four short products (N = 64, so the pipe is never the limit) and a commit; producer:
+// as in test 3, three places in flight.  Background (bounded, ends with the producer): 0 sleeping; 1 four dependent
+// FMA chains per thread; 2 shared-memory load + store; 3 tcgen05.ld x32 + wait back to back; 4 tcgen05.ld x32 + wait,
+// then 32 independent FMA chains, twice (an epilogue-like mix); 5 the same with 64 rounds of arithmetic per load.
+struct BgArgs {
+    long long *out;
+    int *err;
+    int mode, rounds, places;
+    float *sink;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(384, 1) bg_kernel(const __grid_constant__ CUtensorMap map, BgArgs P) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ __align__(8) uint64_t bar[2], lbar[3];
+    __shared__ volatile int stop;
+    __shared__ __align__(16) float scratch[8 * 32 * 8];
+    const uint32_t rank = blockIdx.x & 1u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *g = smem_raw + (base - smem_u32(smem_raw));
+    for (int i = threadIdx.x; i < 2 * SLOT / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(g)[i] = 0x3c003c00u;
+    fence_async_smem();
+    if (threadIdx.x == 0) {
+        stop = 0;
+        mbar_init(smem_u32(&bar[0]), 1);
+        mbar_init(smem_u32(&bar[1]), 1);
+        for (int i = 0; i < 3; ++i) mbar_init(smem_u32(&lbar[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(256u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    if (warp == 1) {
+        if (rank == 0 && elect_one()) {
+            const uint32_t idesc = make_idesc(256, 64);
+            bool ok = true;
+            uint32_t par[2] = {0, 0};
+            const long long c0 = clock64();
+            for (int r = 0; r < P.rounds && ok; ++r) {
+                const int b = r & 1;
+                if (r >= 2) {
+                    ok = wait_bounded(smem_u32(&bar[b]), par[b]);
+                    par[b] ^= 1u;
+                }
+                tc_fence_after();
+                const uint64_t da = make_desc(base), db = make_desc(base + SLOT);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) umma_pair<1>(tmem, da + 2u * i, db + 2u * i, idesc);
+                umma_commit_pair(smem_u32(&bar[b]));
+            }
+            for (int b = 0; b < 2 && ok; ++b) {
+                const int bb = (P.rounds + b) & 1;
+                ok = wait_bounded(smem_u32(&bar[bb]), par[bb]);
+                par[bb] ^= 1u;
+            }
+            P.out[(blockIdx.x >> 1) * 4 + 2] = clock64() - c0;
+            if (!ok) atomicExch(P.err, 1);
+        }
+    } else if (warp == 2) {
+        if (elect_one()) {
+            const uint32_t wbase = base + 2 * SLOT;
+            bool ok = true;
+            uint32_t par = 0;
+            int s = 0, ks = 0, blk = (int)((blockIdx.x * 37u) % 64u);
+            const long long c0 = clock64();
+            for (int r = 0; r < P.places + 3 && ok; ++r) {
+                if (r >= 3) ok = wait_bounded(smem_u32(&lbar[s]), par);
+                if (r < P.places) {
+                    mbar_expect_tx(smem_u32(&lbar[s]), SLOT);
+                    tma_load_2d(wbase + s * SLOT, &map, 64 * ks, 128 * blk, smem_u32(&lbar[s]));
+                    tma_load_2d(wbase + s * SLOT + 8192, &map, 64 * ks, 128 * blk + 64, smem_u32(&lbar[s]));
+                    if (++ks == 9) {
+                        ks = 0;
+                        if (++blk == 64) blk = 0;
+                    }
+                }
+                if (++s == 3) {
+                    s = 0;
+                    if (r >= 3) par ^= 1u;
+                }
+            }
+            if (!ok) atomicExch(P.err, 2);
+            P.out[(blockIdx.x >> 1) * 4 + rank] = clock64() - c0;
+        }
+        __syncwarp();
+        if (lane == 0) stop = 1;  // the background warps of this CTA run until its producer is done
+    } else if (warp >= 4) {
+        float a0 = lane, a1 = lane + 1, a2 = lane + 2, a3 = lane + 3;
+        float v[32];
+        for (int it = 0; it < (1 << 22) && !stop; ++it) {
+            if (P.mode == 1) {
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    a0 = fmaf(a0, 1.0001f, 0.5f);
+                    a1 = fmaf(a1, 0.9999f, 0.25f);
+                    a2 = fmaf(a2, 1.0002f, 0.125f);
+                    a3 = fmaf(a3, 0.9998f, 0.75f);
+                }
+            } else if (P.mode == 2) {
+                float4 *p4 = reinterpret_cast<float4 *>(scratch) + ((warp - 4) * 64 + lane);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float4 x = *p4;
+                    x.x += 1.f;
+                    *p4 = x;
+                    p4 += 32 * ((u & 1) ? -1 : 1);
+                }
+            } else if (P.mode >= 3) {
+                tmem_ld32(tmem + ((uint32_t)(32 * (warp & 3)) << 16) + 64u + 32u * (it & 3), v);
+                tmem_ld_wait();
+                const int reps = P.mode == 3 ? 0 : P.mode == 4 ? 2 : 64;
+                for (int rr = 0; rr < reps; ++rr)
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) v[u] = fmaf(v[u], 1.0001f, 0.5f);
+#pragma unroll
+                for (int u = 0; u < 32; ++u) a0 += v[u];
+            } else {
+                __nanosleep(200);
+            }
+        }
+        if (a0 + a1 + a2 + a3 == 12345.f) P.sink[threadIdx.x] = a0;
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+    }
+}
+
 static bool check(const char *what) {
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -422,6 +564,27 @@ int main() {
                 if (mode) printf(", %.1f cycles per product meanwhile", (double)s[2] / (double)std::max(1LL, s[3]));
                 printf("\n");
             }
+    }
+    {   // ---- 6: the single-thread roles beside working warps
+        const int bsmem = 5 * SLOT + 2048;
+        cudaFuncSetAttribute(bg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bsmem);
+        float *sink;
+        cudaMalloc(&sink, 4096);
+        BgArgs G{out, err, 0, 8192, 4096, sink};
+        const char *names[6] = {"sleeping", "4 dependent FMA chains", "shared-memory load + store", "tcgen05.ld x32 + wait",
+                                "tcgen05.ld + 2 x 32 independent FMA", "tcgen05.ld + 64 x 32 independent FMA"};
+        for (int mode = 0; mode < 6; ++mode) {
+            G.mode = mode;
+            cudaMemset(err, 0, 4);
+            cudaMemset(out, 0, 74 * 4 * 8);
+            bg_kernel<<<2 * 74, 384, bsmem>>>(map, G);
+            if (!check("roles beside working warps")) return 1;
+            long long o4[4];
+            cudaMemcpy(o4, out, 32, cudaMemcpyDeviceToHost);
+            cudaMemcpy(&herr, err, 4, cudaMemcpyDeviceToHost);
+            printf("eight other warps %-38s (err %d): issuer %.0f cycles per round of 4 short products, producer %.0f cycles per place\n",
+                   names[mode], herr, o4[2] / 8192.0, o4[0] / 4096.0);
+        }
     }
     const int osmem = 16 * 8192 + 2048;
     cudaFuncSetAttribute(ops_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, osmem);
