@@ -8,8 +8,8 @@
 // rows 128 r ..: each loads its own rows of the row operand and its half of the tile's weight rows, and the leader
 // issues every product as one tcgen05.mma.cta_group::2 of M = 256, so a weight tile crosses L2 -> shared memory once
 // per 256 rows and a k-step costs each SM 32 KB of loads instead of 48 (the one-CTA form was bound by those loads).
-// Per CTA a TMA producer warp, an MMA warp (the leader's issues) and four epilogue warps; six operand stages and two
-// accumulator buffers; a pair walks several tiles, its epilogue of one under the products of the next.
+// Per CTA two TMA producer warps, an MMA warp (the leader's issues) and eight epilogue warps; five operand stages and
+// two accumulator buffers; a pair walks several tiles, its epilogue of one under the products of the next.
 // Unlike the decode-time encoder, the hidden activations pass through bf16 here (they are an operand of the second
 // product), so a latent written by this path may differ from the fp32-hidden one by a few bf16 ulps of its scale.
 // All waits are bounded and record a code in the status word.
@@ -29,14 +29,15 @@ namespace {
 
 constexpr int PF_M = 128;          // rows per CTA
 constexpr int PF_N = 256;          // columns per CTA at most
-constexpr int PF_STAGES = 6;       // 32 KB each: one CTA per SM
+constexpr int PF_STAGES = 5;       // 32 KB each: one CTA per SM
 constexpr int PF_A_BYTES = PF_M * 128;   // one 64-wide K slab of the row tile (bf16, 128-byte rows)
 constexpr int PF_B_BYTES = (PF_N / 2) * 128;  // this CTA's half of the column tile's weight rows
 constexpr int PF_STAGE_BYTES = PF_A_BYTES + PF_B_BYTES;
-constexpr int PF_EPI_WARPS = 8;    // two per tensor-memory lane quarter: even and odd 32-column groups
+constexpr int PF_EPI_WARPS = 8;    // two per tensor-memory lane quarter: even and odd 64-column blocks
 constexpr int PF_THREADS = 32 * (3 + PF_EPI_WARPS);  // warp 0 producer (row operand), warp 1 MMA + tensor memory,
                                                      // warps 2-9 epilogue, warp 10 producer (weights)
-constexpr int PF_SMEM = PF_STAGES * PF_STAGE_BYTES + 1024 /* alignment */ + 128 /* barriers */;
+constexpr int PF_SMEM = PF_STAGES * PF_STAGE_BYTES + 1024 /* alignment */ + 128 /* barriers */ +
+                        PF_EPI_WARPS * 4096 /* store staging, 32 rows x 128 B per epilogue warp */;
 
 struct PfArgs {
     const EncPlan *plan;         // [2]: K then V (device)
@@ -94,6 +95,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PF_THREADS, 1)
     const uint32_t base = (smem_u32(pf_smem) + 1023u) & ~1023u;
     const uint32_t bars = base + PF_STAGES * PF_STAGE_BYTES;  // full[S] (leader's are used), empty[S], acc_full[2], acc_empty[2]
     const uint32_t bar_accf = bars + 16 * PF_STAGES, bar_acce = bar_accf + 16;
+    const uint32_t stage_base = bars + 128;  // 128-byte aligned (the stages are 1024-byte multiples)
     const int n_slabs = (kdim + 63) >> 6;
     const int n_ct = (ndim + PF_N - 1) / PF_N;
     const int n_tiles = ((a.n_rows_blk + 2 * PF_M - 1) / (2 * PF_M)) * n_ct;
@@ -188,7 +190,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PF_THREADS, 1)
         }
     } else if (warp < 2 + PF_EPI_WARPS) {
         // epilogue: thread = one row of the CTA's half of the tile (tensor-memory lane quarter = warp % 4) and every
-        // other group of 32 columns
+        // other block of 64 columns
         const int q = warp & 3, rl = 32 * q + lane, chalf = (warp - 2) >> 2;
         const uint32_t acce_leader = map_to_cta(bar_acce, 0);
         const float slope = pl.slope;
@@ -230,35 +232,64 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PF_THREADS, 1)
             }
             if (!mbar_wait(bar_accf + 8 * buf, (it >> 1) & 1u, a.status, 0x403)) break;
             tc_fence_after();
-            for (int g = chalf; 32 * g < nt; g += 2) {
-                float v[32];
-                tmem_ld32(acc + ((uint32_t)(32 * q) << 16) + 32u * g, v);
-                tmem_ld_wait();
-                if (!row_ok) continue;
+            // 64 columns (a 128-byte row segment) at a time, the two warps of a lane quarter alternating.  A thread owns a
+            // row, so storing from registers would touch 32 rows with 16 bytes each per instruction; the 32 x 128-byte block
+            // goes through a swizzled staging area of the warp instead and leaves as whole 128-byte lines, four rows per
+            // instruction (lane = 8 l_row + chunk).
+            const uint32_t stg = stage_base + (uint32_t)(warp - 2) * 4096u;
+            const uint64_t dst_bits = reinterpret_cast<uint64_t>(dst);
+            for (int b64 = chalf; 64 * b64 < nt; b64 += 2) {
 #pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    const int c = 32 * g + 8 * c8;
-                    if (c >= nt) break;
-                    float o[8], pa[8], pb[8];
-                    *reinterpret_cast<float4 *>(pa) = *reinterpret_cast<const float4 *>(&prm[0][c]);
-                    *reinterpret_cast<float4 *>(pa + 4) = *reinterpret_cast<const float4 *>(&prm[0][c + 4]);
-                    if (STAGE == 1) {
-                        *reinterpret_cast<float4 *>(pb) = *reinterpret_cast<const float4 *>(&prm[1][c]);
-                        *reinterpret_cast<float4 *>(pb + 4) = *reinterpret_cast<const float4 *>(&prm[1][c + 4]);
-                    }
+                for (int hg = 0; hg < 2; ++hg) {
+                    const int g = 2 * b64 + hg;
+                    if (32 * g >= nt) break;  // warp-uniform
+                    float v[32];
+                    tmem_ld32(acc + ((uint32_t)(32 * q) << 16) + 32u * g, v);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float x = v[8 * c8 + e];
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        const int c = 32 * g + 8 * c8;
+                        if (c >= nt) break;
+                        float o[8], pa[8], pb[8];
+                        *reinterpret_cast<float4 *>(pa) = *reinterpret_cast<const float4 *>(&prm[0][c]);
+                        *reinterpret_cast<float4 *>(pa + 4) = *reinterpret_cast<const float4 *>(&prm[0][c + 4]);
                         if (STAGE == 1) {
-                            const float y = fmaf(x, pa[e], pb[e]);
-                            o[e] = y > 0.f ? y : y * slope;
-                        } else {
-                            o[e] = x + pa[e];
+                            *reinterpret_cast<float4 *>(pb) = *reinterpret_cast<const float4 *>(&prm[1][c]);
+                            *reinterpret_cast<float4 *>(pb + 4) = *reinterpret_cast<const float4 *>(&prm[1][c + 4]);
                         }
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float x = v[8 * c8 + e];
+                            if (STAGE == 1) {
+                                const float y = fmaf(x, pa[e], pb[e]);
+                                o[e] = y > 0.f ? y : y * slope;
+                            } else {
+                                o[e] = x + pa[e];
+                            }
+                        }
+                        const uint32_t chunk = (uint32_t)(4 * hg + c8);  // 16-byte chunk of the row's 128-byte segment
+                        const uint32_t addr = stg + (uint32_t)lane * 128u + ((chunk ^ ((uint32_t)lane & 7u)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(o[0], o[1])),
+                                     "r"(pack_bf16(o[2], o[3])), "r"(pack_bf16(o[4], o[5])), "r"(pack_bf16(o[6], o[7]))
+                                     : "memory");
                     }
-                    *reinterpret_cast<uint4 *>(dst + c) =
-                        make_uint4(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]), pack_bf16(o[4], o[5]), pack_bf16(o[6], o[7]));
                 }
+                __syncwarp();
+                const uint32_t chunk = (uint32_t)lane & 7u;
+                const bool col_ok = 64 * b64 + 8 * (int)chunk < nt;  // widths are multiples of 16: whole chunks
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + (lane >> 3);  // row of the warp's 32
+                    const uint64_t d_row = __shfl_sync(0xffffffffu, dst_bits, rr);
+                    const int ok_row = __shfl_sync(0xffffffffu, (int)row_ok, rr);
+                    uint32_t w0, w1, w2, w3;
+                    const uint32_t addr = stg + (uint32_t)rr * 128u + ((chunk ^ ((uint32_t)rr & 7u)) << 4);
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(addr) : "memory");
+                    if (ok_row && col_ok)
+                        *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(d_row) + 64 * b64 + 8 * (int)chunk) =
+                            make_uint4(w0, w1, w2, w3);
+                }
+                __syncwarp();  // the staging area is free for the next block
             }
             // this warp is done reading the buffer: one arrival of the sixteen the issuer waits for
             tc_fence_before();
