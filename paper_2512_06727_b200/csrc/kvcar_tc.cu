@@ -998,37 +998,28 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                         float y[64];
                         tmem_ld32(acc + 64u * hp, y);
                         tmem_ld32(acc + 64u * hp + 32u, y + 32);
-                        // q . (k' + b) = q . k' + q . b: the bias term is one number per query head, formed by the warp
-                        // (two channels per lane) while the accumulator loads are in flight
-                        const float *bh = b2 + job_slot(job, hp) * 64;
-                        const int ql0 = (job_kvh(job, hp) - h_lo) * group;
-                        float qb[2] = {0.f, 0.f};  // this build serves groups of one or two query heads
-#pragma unroll
-                        for (int g = 0; g < 2; ++g)
-                            if (g < group) {
-                                const float *qh = qs + (ql0 + g) * 64;
-                                float p = fmaf(qh[lane], bh[lane], qh[lane + 32] * bh[lane + 32]);
-#pragma unroll
-                                for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
-                                qb[g] = p;
-                            }
                         tmem_ld_wait();
+                        const float4 *bb = reinterpret_cast<const float4 *>(b2 + job_slot(job, hp) * 64);
+                        float2 y2[32];
 #pragma unroll
-                        for (int g = 0; g < 2; ++g)
-                            if (g < group) {
-                                const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g) * 64);
-                                float2 d0 = make_float2(0.f, 0.f), d1 = d0, d2 = d0, d3 = d0;  // four chains
+                        for (int c = 0; c < 16; ++c) {
+                            const float4 b4 = bb[c];
+                            y2[2 * c] = __fadd2_rn(make_float2(y[4 * c], y[4 * c + 1]), make_float2(b4.x, b4.y));
+                            y2[2 * c + 1] = __fadd2_rn(make_float2(y[4 * c + 2], y[4 * c + 3]), make_float2(b4.z, b4.w));
+                        }
+                        const int ql0 = (job_kvh(job, hp) - h_lo) * group;
+                        for (int g = 0; g < group; ++g) {
+                            const float4 *q4 = reinterpret_cast<const float4 *>(qs + (ql0 + g) * 64);
+                            float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
 #pragma unroll
-                                for (int c = 0; c < 16; c += 2) {
-                                    const float4 qa = q4[c], qc = q4[c + 1];
-                                    d0 = __ffma2_rn(make_float2(y[4 * c], y[4 * c + 1]), make_float2(qa.x, qa.y), d0);
-                                    d1 = __ffma2_rn(make_float2(y[4 * c + 2], y[4 * c + 3]), make_float2(qa.z, qa.w), d1);
-                                    d2 = __ffma2_rn(make_float2(y[4 * c + 4], y[4 * c + 5]), make_float2(qc.x, qc.y), d2);
-                                    d3 = __ffma2_rn(make_float2(y[4 * c + 6], y[4 * c + 7]), make_float2(qc.z, qc.w), d3);
-                                }
-                                const float dot = ((d0.x + d0.y) + (d1.x + d1.y)) + ((d2.x + d2.y) + (d3.x + d3.y)) + qb[g];
-                                Smine[(ql0 + g) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
+                            for (int c = 0; c < 16; ++c) {
+                                const float4 qq = q4[c];
+                                d0 = __ffma2_rn(y2[2 * c], make_float2(qq.x, qq.y), d0);
+                                d1 = __ffma2_rn(y2[2 * c + 1], make_float2(qq.z, qq.w), d1);
                             }
+                            const float dot = (d0.x + d0.y) + (d1.x + d1.y);
+                            Smine[(ql0 + g) * PSTRIDE + row] = row < mine.valid ? dot : -INFINITY;
+                        }
                     }
                     tc_fence_before();
                     __syncwarp();
