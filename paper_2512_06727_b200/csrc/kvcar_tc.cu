@@ -1180,9 +1180,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                             float dv[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                             for (int gi = 0; gi < 4; ++gi) {
                                 if (32 * gi >= tt.valid) break;
-                                uint32_t r[2][16];
-                                tmem_ld_frag_x4(acc + 128u * chalf + 32u * gi, r[0]);
-                                tmem_ld_frag_x4(acc + (16u << 16) + 128u * chalf + 32u * gi, r[1]);
                                 uint32_t bp[4];
 #pragma unroll
                                 for (int ks = 0; ks < 2; ++ks) {
@@ -1190,6 +1187,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
                                     bp[2 * ks] = n < group ? *reinterpret_cast<const uint32_t *>(pr) : 0u;
                                     bp[2 * ks + 1] = n < group ? *reinterpret_cast<const uint32_t *>(pr + 8) : 0u;
                                 }
+                                // nothing between the tensor-memory loads and their wait: until then the destination
+                                // registers are written behind the compiler's back, and code placed in between gives it
+                                // reasons to move them
+                                uint32_t r[2][16];
+                                tmem_ld_frag_x4(acc + 128u * chalf + 32u * gi, r[0]);
+                                tmem_ld_frag_x4(acc + (16u << 16) + 128u * chalf + 32u * gi, r[1]);
                                 tmem_ld_wait();
                                 if (32 * gi + 32 > tt.valid) {  // rows past the tile's end may hold anything
 #pragma unroll

@@ -123,3 +123,43 @@ def test_config3_uncompressed_twin_sampled():
     the lower layer's rows): the streaming kernel with 8 query heads per KV head."""
     w = synth.scaled(synth.CONFIGS["c3"], n_layers=6)
     _run(w, [5, 31], steps=1, compress=False)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("cfg,batch", [("c5", 256), ("c3", 32)])
+def test_fused_steps_back_to_back_equal_the_same_steps_synchronised(cfg, batch):
+    """Three decode steps of the whole stack through kvcar_step_layer with nothing between the calls (the tile kernel
+    of one layer on the side stream, the next layer's encoder behind it: how a serving loop and the bench drive the
+    library), against the same three steps on a second, identically filled context with a device synchronise after
+    every layer: no device error, guard regions intact, outputs bit-equal.  The element-wise parity tests synchronise
+    per layer (they copy every output back), so only this test sees the launches overlap at full size."""
+    import bench
+    w = synth.scaled(synth.CONFIGS[cfg], batch=batch)
+
+    class A:
+        pass
+    outs = []
+    for synchronise in (False, True):
+        a2 = A()
+        a2.uncompressed = False
+        a2.kernel = "auto"
+        sess, src, aes = bench.build_session(w, a2, torch, 3 + 24)
+        sess.has_autoencoders = bool(aes)
+        bench.fast_prefill(sess, w, torch)
+        seqs = list(range(w.batch))
+        stream = sess.stream()
+        k, v, q, out = bench.step_inputs(sess, w, torch, 3)
+        for i in range(3):
+            for l in range(w.n_layers):
+                sess.ctx.step_layer(l, seqs, k[i, l].data_ptr(), v[i, l].data_ptr(), q[i, l].data_ptr(),
+                                    out[i, l].data_ptr(), B.INCLUDE_CURRENT_EXACT, stream)
+                if synchronise:
+                    torch.cuda.synchronize()
+            sess.ctx.advance(seqs, 1, stream)
+        torch.cuda.synchronize()
+        sess.ctx.sync_status(stream)
+        assert sess.ctx.debug_check(stream) == (0, 0, -1)
+        assert bool(torch.isfinite(out.float()).all())
+        outs.append(out.clone())
+        del sess
+    assert torch.equal(outs[0], outs[1])
