@@ -248,8 +248,11 @@ kvcar_status kvcar_step_layer(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs
  * The same step for one layer with HOST buffers: copies k, v, q (each
  * n_tokens = 1) to the device, runs kvcar_step_layer, and copies `out`
  * back, all ordered on `stream`.  Returns
- * after enqueuing; synchronise the stream before reading out_host.  Host
- * buffers should be page-locked for the copies to be asynchronous.
+ * after enqueuing; synchronise the stream before reading out_host.  k, v
+ * and q are gathered into one of eight page-locked slots of the context and
+ * cross in a single copy (the call waits for the copy that used the slot eight
+ * calls earlier), so k_host, v_host and q_host may be reused as soon as the
+ * call returns; out_host should be page-locked for its copy to be asynchronous.
  */
 kvcar_status kvcar_step_layer_host(kvcar_ctx *ctx, int32_t layer, const int32_t *seqs, int32_t n_seqs,
                                    const void *k_host, const void *v_host, const void *q_host, void *out_host,

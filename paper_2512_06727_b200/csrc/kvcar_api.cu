@@ -52,6 +52,14 @@ struct kvcar_ctx {
     // kvcar_step_layer runs the tile kernel beside the encoder: a stream and two events of the library's own
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // kvcar_step_layer_host: pinned host slots in which a call's k, v and q are laid out as on the device, so that they
+    // cross in one copy; a slot is reused once the copy that read it last has completed (its event)
+    static constexpr int H_SLOTS = 8;
+    char *hstage = nullptr;
+    size_t hslot_bytes = 0;
+    cudaEvent_t ev_h[H_SLOTS] = {};
+    bool ev_h_used[H_SLOTS] = {};
+    unsigned hslot = 0;
 
     // pages
     std::vector<int32_t> free_pages;
@@ -373,6 +381,9 @@ kvcar_status kvcar_destroy(kvcar_ctx *ctx) {
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->side) cudaStreamDestroy(ctx->side);
+    for (cudaEvent_t e : ctx->ev_h)
+        if (e) cudaEventDestroy(e);
+    if (ctx->hstage) cudaFreeHost(ctx->hstage);
     delete ctx;
     return KVCAR_OK;
 }
@@ -633,6 +644,19 @@ kvcar_status kvcar_bind_memory(kvcar_ctx *c, void *pool, size_t pool_bytes, void
         float *p = nullptr;
         if (static_scratch_for_current_device(&p) != cudaSuccess) cudaGetLastError();
         c->static_scratch = p;
+    }
+    if (!c->hstage) {  // set-up time: the host-buffer entry point's staging slots (without them it copies k, v, q singly)
+        const size_t nbatch = (size_t)std::min(g.max_seqs, KVCAR_MAX_BATCH);
+        const size_t kvb = align_up(nbatch * hkv * hd * c->elem, 256), qb = align_up(nbatch * g.n_q_heads * hd * c->elem, 256);
+        c->hslot_bytes = 2 * kvb + qb;
+        bool ok = cudaHostAlloc((void **)&c->hstage, c->hslot_bytes * kvcar_ctx::H_SLOTS, cudaHostAllocDefault) == cudaSuccess;
+        for (int i = 0; ok && i < kvcar_ctx::H_SLOTS; ++i)
+            ok = cudaEventCreateWithFlags(&c->ev_h[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            if (c->hstage) cudaFreeHost(c->hstage);
+            c->hstage = nullptr;
+        }
     }
     for (size_t off : c->guard_off)
         if (cudaMemsetAsync(c->pool + off, GUARD_FILL, GUARD_BYTES, st) != cudaSuccess)
@@ -953,12 +977,28 @@ kvcar_status kvcar_step_layer_host(kvcar_ctx *c, int32_t layer, const int32_t *s
     const size_t qb = align_up((size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, 256);
     char *dk = c->ws + c->stage_off, *dv = dk + kvb, *dq = dv + kvb, *dout = dq + qb;
     cudaStream_t st = (cudaStream_t)stream;
-    cudaError_t e = cudaMemcpyAsync(dk, k_host, (size_t)n_seqs * g.n_kv_heads * g.head_dim * c->elem,
-                                    cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(dv, v_host, (size_t)n_seqs * g.n_kv_heads * g.head_dim * c->elem, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(dq, q_host, (size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem, cudaMemcpyHostToDevice, st);
+    const size_t kv_bytes = (size_t)n_seqs * g.n_kv_heads * g.head_dim * c->elem;
+    const size_t q_bytes = (size_t)n_seqs * g.n_q_heads * g.head_dim * c->elem;
+    cudaError_t e;
+    if (c->hstage && 2 * kvb + q_bytes <= c->hslot_bytes) {
+        // one copy: k, v, q gathered in a pinned slot with the device staging area's layout
+        const unsigned slot = c->hslot++ % kvcar_ctx::H_SLOTS;
+        if (c->ev_h_used[slot]) {
+            e = cudaEventSynchronize(c->ev_h[slot]);  // the copy that read this slot eight calls ago
+            if (e != cudaSuccess) return cuda_fail(c, e, "staging slot");
+        }
+        char *h = c->hstage + (size_t)slot * c->hslot_bytes;
+        memcpy(h, k_host, kv_bytes);
+        memcpy(h + kvb, v_host, kv_bytes);
+        memcpy(h + 2 * kvb, q_host, q_bytes);
+        e = cudaMemcpyAsync(dk, h, 2 * kvb + q_bytes, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_h[slot], st);
+        c->ev_h_used[slot] = e == cudaSuccess;
+    } else {
+        e = cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, st);
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "host to device copy");
     kvcar_status s = kvcar_step_layer(c, layer, seqs, n_seqs, dk, dv, dq, dout, flags, stream);
     if (s != KVCAR_OK) return s;
