@@ -279,3 +279,17 @@ def test_trace_report_reads_synthetic_stamps(capsys):
     trace.report({"0.2": [], "0.3": []}, 5)
     assert "no stamps" in capsys.readouterr().out
 
+
+
+def test_status_codes_of_the_header_match_the_binding():
+    """Every KVCAR_ERR_* / KVCAR_OK of include/kvcar.h has the same number and name in the Python binding (a status the
+    binding cannot name would be raised as a bare number)."""
+    import os
+    import re
+    from paper_2512_06727_b200 import binding as B
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    text = open(os.path.join(root, "include", "kvcar.h")).read()
+    body = text[text.index("KVCAR_OK = 0"):]
+    body = body[:body.index("}")]
+    codes = {int(v): k for k, v in re.findall(r"KVCAR_(?:ERR_)?([A-Z_]+)\s*=\s*(\d+)", body)}
+    assert codes == B.STATUS_NAMES, (codes, B.STATUS_NAMES)
